@@ -1,0 +1,203 @@
+/*
+ * mnn_conv.h — C ABI of the B200 (sm_100a) convolution library.
+ *
+ * The library computes y = act(conv2d(x, w) + bias) on NCHW fp32 tensors through
+ * one of three schemes chosen ahead of inference (the paper's "pre-inference",
+ * Section 3.2): Winograd F(m x m, k x k) (Eq. 6), a GEMM over gathered patches
+ * (k = 1 "is just a matrix multiplication", Section 3.2 item 1; k > 1 strided or
+ * dilated layers gather patches first) and a direct "sliding window" kernel
+ * (Section 3.2 item 3, Eq. 3).
+ *
+ * Conventions for every entry point
+ *   - x, w, bias, y and the workspace are DEVICE pointers owned by the caller,
+ *     dense and contiguous: x [N][Cin][H][W], w [Cout][Cin/groups][k][k],
+ *     bias [Cout] (NULL = zeros), y [N][Cout][OH][OW], all fp32 and 16-byte aligned.
+ *   - OH = floor((H + 2 pad - dilation (k-1) - 1)/stride) + 1, same for OW.
+ *     Cross-correlation (no kernel flip).
+ *   - Matrices and info structs are HOST pointers.
+ *   - `stream` is a cudaStream_t passed as void*.  Runs are asynchronous on it;
+ *     the library never synchronises and never allocates device memory in a run.
+ *   - Functions returning int give MNN_OK (0) or a negative mnn_status; the reason
+ *     is kept in a thread-local string read with mnn_last_error().
+ *   - A plan is immutable after creation and may be used from one stream at a
+ *     time (its workspace is per plan).  y must not alias x.
+ *   - There is no CPU fallback: without a CUDA device runs fail with MNN_ECUDA.
+ */
+#ifndef MNN_CONV_H_
+#define MNN_CONV_H_
+
+#if defined(__GNUC__)
+#define MNN_API __attribute__((visibility("default")))
+#else
+#define MNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mnn_conv_plan_s* mnn_conv_plan_t;   /* opaque host object */
+
+typedef enum {
+    MNN_OK = 0,
+    MNN_EINVAL = -1,         /* argument outside the definition (NULL, non-positive size, ...) */
+    MNN_EUNSUPPORTED = -2,   /* valid but not implemented (e.g. forced Winograd with stride 2) */
+    MNN_EWORKSPACE = -3,     /* workspace missing or too small */
+    MNN_EALIGN = -4,         /* a device pointer is not 16-byte aligned */
+    MNN_ECUDA = -5,          /* a CUDA call failed, or a kernel reported a bounded wait that ran out */
+    MNN_ENOTCALIBRATED = -6
+} mnn_status;
+
+enum { MNN_ALGO_AUTO = 0, MNN_ALGO_WINOGRAD = 1, MNN_ALGO_GEMM = 2, MNN_ALGO_DIRECT = 3 };
+enum { MNN_PREC_TF32 = 0, MNN_PREC_BF16 = 1 };             /* accuracy class */
+enum { MNN_OPERAND_AUTO = 0, MNN_OPERAND_TF32 = 1, MNN_OPERAND_BF16 = 2, MNN_OPERAND_FP32_REF = 3 };
+enum { MNN_POINTS_AUTO = 0, MNN_POINTS_PAPER = 1, MNN_POINTS_UNIT = 2, MNN_POINTS_MIXED = 3 };
+enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_STAGE_OUTPUT = 8,
+       MNN_STAGE_ALL = 15 };
+
+#define MNN_N_CANDIDATES 16
+#define MNN_N_CONSTS 16
+#define MNN_COST_INADMISSIBLE 0xFFFFFFFFFFFFFFFFull
+
+/*
+ * Options of mnn_conv_plan_ex.  Zero-initialise for the defaults of mnn_conv_plan
+ * except `relu`, which mnn_conv_plan sets to 1.
+ *   groups     1, or Cin (= Cout) for a depthwise layer.  0 means 1.
+ *   relu       0/1: y = max(0, .) after the bias.
+ *   precision  accuracy class the result must meet against an exact evaluation:
+ *              MNN_PREC_TF32: relative L2 error <= 1e-3; MNN_PREC_BF16: <= 1e-2.
+ *   operand    tensor-core operand format of the contraction; AUTO lets the
+ *              planner pick any format/pass count admissible for the class.
+ *              FP32_REF runs the contraction on CUDA cores in fp32 (a slow
+ *              checking path, never chosen by the planner).
+ *   passes     0 = planner; 1 = operands rounded once; 3 = each operand split
+ *              into hi + lo of the operand format and hi*hi + lo*hi + hi*lo
+ *              accumulated (near-fp32 accuracy at 3x the tensor work).
+ *   force_algo MNN_ALGO_*; AUTO = planner.
+ *   force_m    0 = planner, else the Winograd output tile size m (2..8).
+ *   points_id  interpolation point set of the generator (Eq. 8): PAPER = 0, +-1/2,
+ *              +-1, ... (the paper's f = 1/2); UNIT = 0, +-1, +-2, ...; MIXED = 0, +-1,
+ *              +-1/2, +-2, +-1/4, +-4; AUTO = the set with the lowest predicted error.
+ *   chunk_images  0 = planner; else images per pipeline chunk (the batch is cut so
+ *              that the transformed tensors of one chunk stay in L2).
+ */
+typedef struct {
+    int groups;
+    int relu;
+    int precision;
+    int operand;
+    int passes;
+    int force_algo;
+    int force_m;
+    int points_id;
+    int chunk_images;
+    int reserved[7];
+} mnn_conv_opts;
+
+/*
+ * What the planner decided (Eq. 1-5 re-stated for this GPU: per candidate
+ * cost = sum over its kernels of max(bytes * c_byte, tensor flops * c_tensor,
+ * ALU flops * c_alu) + launch cost, in integer picoseconds).
+ * cost_ps[] order: 0 DIRECT; 1 GEMM tf32; 2 GEMM bf16; 3..5 Winograd m=2,4,6 tf32x1;
+ * 6..8 tf32x3; 9..11 bf16x1; 12..14 bf16x3; 15 unused.  Candidates that are not
+ * applicable or fail the accuracy gate hold MNN_COST_INADMISSIBLE.
+ * Workspace layout (byte offsets from the workspace base, each 1024-aligned):
+ *   u_offset  transformed weights  U [alpha^2][Cout][cin_pad]  (operand format; hi then lo when passes = 3)
+ *   v_offset  transformed inputs   V [alpha^2][chunk_tiles][cin_pad] of one chunk (same format)
+ *   m_offset  contraction results  M [alpha^2][Cout][m_row_stride] fp32 of one chunk
+ * For the GEMM scheme alpha = 1, cin_pad covers Cin*k*k and M is unused.
+ */
+typedef struct {
+    int algo, m, alpha, precision, operand, passes, points_id;
+    int OH, OW, groups, relu;
+    int chunk_images, n_chunks, launches_per_run;
+    int cin_pad, m_row_stride;
+    long long chunk_tiles;           /* Winograd tiles (or GEMM columns) per full chunk */
+    long long workspace_bytes;       /* total the caller must provide (0 for DIRECT) */
+    long long u_offset, u_bytes, v_offset, v_bytes, m_offset, m_bytes;
+    long long predicted_error_ppm;   /* accuracy model's relative L2 error x 1e6 for the choice */
+    int chosen_candidate;            /* index into cost_ps, -1 when the choice was forced outside the list */
+    int reserved;
+    unsigned long long cost_ps[MNN_N_CANDIDATES];
+} mnn_conv_info;
+
+/* Plan one layer with groups = 1, relu = 1, accuracy class TF32, everything else
+ * decided by the planner (Section 3.2 "computation scheme selection").  Host only;
+ * needs no GPU.  Returns NULL on error. */
+MNN_API mnn_conv_plan_t mnn_conv_plan(int N, int Cin, int Cout, int H, int W, int k,
+                              int stride, int pad, int dilation);
+
+/* Same with explicit options (opts may be NULL = all defaults incl. relu = 0). */
+MNN_API mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k,
+                                 int stride, int pad, int dilation, const mnn_conv_opts* opts);
+
+/* Copy the plan's decisions into *info (host). */
+MNN_API int mnn_conv_plan_query(mnn_conv_plan_t plan, mnn_conv_info* info);
+
+/* Hand the plan its device workspace (>= info.workspace_bytes, 1024-byte aligned).
+ * The caller keeps ownership and must keep it alive while the plan is used
+ * (memory pre-allocation ahead of inference, Section 3.2 "preparation-execution
+ * decoupling").  Invalidates prepared weights. */
+MNN_API int mnn_conv_set_workspace(mnn_conv_plan_t plan, void* workspace, long long bytes);
+
+/* Transform the weights into the workspace now (U = G w G^T of Eq. 6, or the
+ * rounded copy the GEMM scheme uses).  Optional: mnn_conv_run does it on first
+ * use of a given w pointer.  Asynchronous on stream. */
+MNN_API int mnn_conv_prepare_weights(mnn_conv_plan_t plan, const float* w, void* stream);
+
+/* One forward pass of the layer: y = act(conv(x, w) + bias).  If w differs from
+ * the pointer last prepared, the weight transform runs first on the stream. */
+MNN_API int mnn_conv_run(mnn_conv_plan_t plan, const float* x, const float* w, const float* bias,
+                 float* y, void* stream);
+
+/* The same pass restricted to the stages in stage_mask (MNN_STAGE_*), for checking
+ * and timing the stages one by one: INPUT writes V (Eq. 6, B^T X B), CONTRACT reads
+ * U, V and writes M (Section 3.3.1 (2): the Hadamard product summed over channels as
+ * one matrix product per transform position), OUTPUT reads M and writes y (A^T . A,
+ * plus bias and ReLU).  Each selected stage runs for every chunk.  For GEMM plans
+ * INPUT is the patch gather and CONTRACT writes y; DIRECT plans have one stage
+ * (MNN_STAGE_CONTRACT). */
+MNN_API int mnn_conv_run_stages(mnn_conv_plan_t plan, const float* x, const float* w, const float* bias,
+                        float* y, void* stream, unsigned stage_mask);
+
+/* Read and clear the device-side status word of the plan (synchronises the
+ * stream): 0 = no kernel reported a problem; otherwise a code naming the bounded
+ * wait that ran out.  Returns MNN_OK and stores the code in *code. */
+MNN_API int mnn_conv_device_status(mnn_conv_plan_t plan, void* stream, int* code);
+
+MNN_API void mnn_conv_destroy(mnn_conv_plan_t plan);
+
+/* Winograd generator (Eq. 8): transform matrices of F(m, k) from the chosen
+ * interpolation points plus the point at infinity, computed in exact rational
+ * arithmetic and rounded once to fp32.  Host arrays, row-major:
+ * At [m][alpha], G [alpha][k], Bt [alpha][alpha], alpha = m + k - 1 <= 16.
+ * Any may be NULL.  points_id must not be AUTO. */
+MNN_API int mnn_winograd_matrices(int m, int k, int points_id, float* At, float* G, float* Bt);
+
+/* Predicted relative L2 error x 1e6 of Winograd F(m,k) with the given point set,
+ * operand format (MNN_OPERAND_TF32/BF16) and passes (1/3): a deterministic host
+ * simulation with rounded operands; the planner's accuracy gate.  m = 1 with
+ * points_id = 0 gives the figure of the GEMM scheme (no transforms).  < 0 on error. */
+MNN_API long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int passes);
+
+/* Cost-model constants (Eq. 5's FLOPS and t_schedule, re-stated for this GPU).
+ * consts[0] attoseconds per HBM byte          consts[1] attoseconds per L2-resident byte
+ * consts[2] attoseconds per TF32 tensor flop  consts[3] attoseconds per BF16 tensor flop
+ * consts[4] attoseconds per fp32 ALU flop     consts[5] picoseconds per kernel launch
+ * consts[6] L2 bytes usable for one chunk     consts[7] number of SMs
+ * consts[8] attoseconds per flop of the direct kernel
+ * consts[9..15] reserved (0).
+ * mnn_calibrate measures them on the current device (launches micro-benchmarks and
+ * synchronises; allocates and frees its own scratch) and installs them;
+ * mnn_set_calibration installs a frozen record so that plans are reproducible;
+ * mnn_get_calibration reads the record in force (built-in defaults if none was set). */
+MNN_API int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CONSTS]);
+MNN_API int mnn_set_calibration(const long long consts[MNN_N_CONSTS]);
+MNN_API int mnn_get_calibration(long long consts[MNN_N_CONSTS]);
+
+MNN_API const char* mnn_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MNN_CONV_H_ */

@@ -1,0 +1,262 @@
+"""ctypes face of the C-ABI library (``include/mnn_conv.h``): same names, argument
+marshalling only.  PyTorch appears only in :class:`ConvLayerRunner`, which uses it
+for device memory and the current stream; every step of the path runs in the
+library's kernels.  There is no fallback: if the shared library is missing,
+loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmnnconv_b200.so")
+
+MNN_OK, MNN_EINVAL, MNN_EUNSUPPORTED, MNN_EWORKSPACE, MNN_EALIGN, MNN_ECUDA, MNN_ENOTCALIBRATED = 0, -1, -2, -3, -4, -5, -6
+ALGO_AUTO, ALGO_WINOGRAD, ALGO_GEMM, ALGO_DIRECT = 0, 1, 2, 3
+PREC_TF32, PREC_BF16 = 0, 1
+OPERAND_AUTO, OPERAND_TF32, OPERAND_BF16, OPERAND_FP32_REF = 0, 1, 2, 3
+POINTS_AUTO, POINTS_PAPER, POINTS_UNIT, POINTS_MIXED = 0, 1, 2, 3
+STAGE_WEIGHT, STAGE_INPUT, STAGE_CONTRACT, STAGE_OUTPUT, STAGE_ALL = 1, 2, 4, 8, 15
+N_CANDIDATES, N_CONSTS = 16, 16
+COST_INADMISSIBLE = 0xFFFFFFFFFFFFFFFF
+ALGO_NAMES = {ALGO_WINOGRAD: "winograd", ALGO_GEMM: "gemm", ALGO_DIRECT: "direct"}
+OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "fp32ref", 0: "-"}
+
+EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_query", "mnn_conv_set_workspace",
+            "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
+            "mnn_conv_destroy", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
+            "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error"]
+
+
+class ConvOpts(ctypes.Structure):
+    _fields_ = [("groups", ctypes.c_int), ("relu", ctypes.c_int), ("precision", ctypes.c_int),
+                ("operand", ctypes.c_int), ("passes", ctypes.c_int), ("force_algo", ctypes.c_int),
+                ("force_m", ctypes.c_int), ("points_id", ctypes.c_int), ("chunk_images", ctypes.c_int),
+                ("reserved", ctypes.c_int * 7)]
+
+
+class ConvInfo(ctypes.Structure):
+    _fields_ = [("algo", ctypes.c_int), ("m", ctypes.c_int), ("alpha", ctypes.c_int), ("precision", ctypes.c_int),
+                ("operand", ctypes.c_int), ("passes", ctypes.c_int), ("points_id", ctypes.c_int),
+                ("OH", ctypes.c_int), ("OW", ctypes.c_int), ("groups", ctypes.c_int), ("relu", ctypes.c_int),
+                ("chunk_images", ctypes.c_int), ("n_chunks", ctypes.c_int), ("launches_per_run", ctypes.c_int),
+                ("cin_pad", ctypes.c_int), ("m_row_stride", ctypes.c_int),
+                ("chunk_tiles", ctypes.c_longlong), ("workspace_bytes", ctypes.c_longlong),
+                ("u_offset", ctypes.c_longlong), ("u_bytes", ctypes.c_longlong),
+                ("v_offset", ctypes.c_longlong), ("v_bytes", ctypes.c_longlong),
+                ("m_offset", ctypes.c_longlong), ("m_bytes", ctypes.c_longlong),
+                ("predicted_error_ppm", ctypes.c_longlong),
+                ("chosen_candidate", ctypes.c_int), ("reserved", ctypes.c_int),
+                ("cost_ps", ctypes.c_ulonglong * N_CANDIDATES)]
+
+
+class MnnError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__("mnn_conv error %d: %s" % (code, message))
+        self.code = code
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library (raises OSError if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise OSError("%s is missing: run `python -m paper_2002_12418_b200.build`" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        i, p, ll = ctypes.c_int, ctypes.c_void_p, ctypes.c_longlong
+        L.mnn_conv_plan.argtypes = [i] * 9
+        L.mnn_conv_plan.restype = p
+        L.mnn_conv_plan_ex.argtypes = [i] * 9 + [ctypes.POINTER(ConvOpts)]
+        L.mnn_conv_plan_ex.restype = p
+        L.mnn_conv_plan_query.argtypes = [p, ctypes.POINTER(ConvInfo)]
+        L.mnn_conv_plan_query.restype = i
+        L.mnn_conv_set_workspace.argtypes = [p, p, ll]
+        L.mnn_conv_set_workspace.restype = i
+        L.mnn_conv_prepare_weights.argtypes = [p, p, p]
+        L.mnn_conv_prepare_weights.restype = i
+        L.mnn_conv_run.argtypes = [p, p, p, p, p, p]
+        L.mnn_conv_run.restype = i
+        L.mnn_conv_run_stages.argtypes = [p, p, p, p, p, p, ctypes.c_uint]
+        L.mnn_conv_run_stages.restype = i
+        L.mnn_conv_device_status.argtypes = [p, p, ctypes.POINTER(i)]
+        L.mnn_conv_device_status.restype = i
+        L.mnn_conv_destroy.argtypes = [p]
+        L.mnn_conv_destroy.restype = None
+        L.mnn_winograd_matrices.argtypes = [i, i, i, p, p, p]
+        L.mnn_winograd_matrices.restype = i
+        L.mnn_accuracy_ppm.argtypes = [i] * 5
+        L.mnn_accuracy_ppm.restype = ll
+        L.mnn_calibrate.argtypes = [i, p, ctypes.POINTER(ll)]
+        L.mnn_calibrate.restype = i
+        L.mnn_set_calibration.argtypes = [ctypes.POINTER(ll)]
+        L.mnn_set_calibration.restype = i
+        L.mnn_get_calibration.argtypes = [ctypes.POINTER(ll)]
+        L.mnn_get_calibration.restype = i
+        L.mnn_last_error.argtypes = []
+        L.mnn_last_error.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def mnn_last_error() -> str:
+    return (lib().mnn_last_error() or b"").decode()
+
+
+def _check(rc: int) -> None:
+    if rc != MNN_OK:
+        raise MnnError(rc, mnn_last_error())
+
+
+def make_opts(groups=1, relu=0, precision=PREC_TF32, operand=0, passes=0, force_algo=0, force_m=0, points_id=0,
+              chunk_images=0) -> ConvOpts:
+    o = ConvOpts()
+    o.groups, o.relu, o.precision, o.operand, o.passes = groups, int(bool(relu)), precision, operand, passes
+    o.force_algo, o.force_m, o.points_id, o.chunk_images = force_algo, force_m, points_id, chunk_images
+    return o
+
+
+def mnn_conv_plan(N, Cin, Cout, H, W, k, stride, pad, dilation):
+    h = lib().mnn_conv_plan(N, Cin, Cout, H, W, k, stride, pad, dilation)
+    if not h:
+        raise MnnError(MNN_EINVAL, mnn_last_error())
+    return h
+
+
+def mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation, opts: ConvOpts | None):
+    h = lib().mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation,
+                               ctypes.byref(opts) if opts is not None else None)
+    if not h:
+        raise MnnError(MNN_EINVAL, mnn_last_error())
+    return h
+
+
+def mnn_conv_plan_query(plan) -> ConvInfo:
+    info = ConvInfo()
+    _check(lib().mnn_conv_plan_query(plan, ctypes.byref(info)))
+    return info
+
+
+def mnn_conv_set_workspace(plan, ptr: int, nbytes: int) -> None:
+    _check(lib().mnn_conv_set_workspace(plan, ptr, nbytes))
+
+
+def mnn_conv_prepare_weights(plan, w_ptr: int, stream: int) -> None:
+    _check(lib().mnn_conv_prepare_weights(plan, w_ptr, stream))
+
+
+def mnn_conv_run(plan, x_ptr: int, w_ptr: int, bias_ptr, y_ptr: int, stream: int) -> None:
+    _check(lib().mnn_conv_run(plan, x_ptr, w_ptr, bias_ptr, y_ptr, stream))
+
+
+def mnn_conv_run_stages(plan, x_ptr, w_ptr, bias_ptr, y_ptr, stream: int, stage_mask: int) -> None:
+    _check(lib().mnn_conv_run_stages(plan, x_ptr, w_ptr, bias_ptr, y_ptr, stream, stage_mask))
+
+
+def mnn_conv_device_status(plan, stream: int) -> int:
+    code = ctypes.c_int(0)
+    _check(lib().mnn_conv_device_status(plan, stream, ctypes.byref(code)))
+    return code.value
+
+
+def mnn_conv_destroy(plan) -> None:
+    lib().mnn_conv_destroy(plan)
+
+
+def mnn_winograd_matrices(m: int, k: int, points_id: int):
+    """(At [m x alpha], G [alpha x k], Bt [alpha x alpha]) as nested lists of fp32 values."""
+    alpha = m + k - 1
+    At = (ctypes.c_float * (m * alpha))()
+    G = (ctypes.c_float * (alpha * k))()
+    Bt = (ctypes.c_float * (alpha * alpha))()
+    _check(lib().mnn_winograd_matrices(m, k, points_id, At, G, Bt))
+    rows = lambda a, r, c: [[a[i * c + j] for j in range(c)] for i in range(r)]
+    return rows(At, m, alpha), rows(G, alpha, k), rows(Bt, alpha, alpha)
+
+
+def mnn_accuracy_ppm(m, k, points_id, operand, passes) -> int:
+    v = lib().mnn_accuracy_ppm(m, k, points_id, operand, passes)
+    if v < 0:
+        raise MnnError(MNN_EINVAL, mnn_last_error())
+    return int(v)
+
+
+def mnn_calibrate(device: int, stream: int) -> list[int]:
+    c = (ctypes.c_longlong * N_CONSTS)()
+    _check(lib().mnn_calibrate(device, stream, c))
+    return list(c)
+
+
+def mnn_set_calibration(consts) -> None:
+    c = (ctypes.c_longlong * N_CONSTS)(*list(consts))
+    _check(lib().mnn_set_calibration(c))
+
+
+def mnn_get_calibration() -> list[int]:
+    c = (ctypes.c_longlong * N_CONSTS)()
+    _check(lib().mnn_get_calibration(c))
+    return list(c)
+
+
+class ConvLayerRunner:
+    """A plan plus its torch-owned workspace.  ``run`` launches on torch's current
+    stream through mnn_conv_run; nothing here computes."""
+
+    def __init__(self, N, Cin, Cout, H, W, k, stride=1, pad=0, dilation=1, opts: ConvOpts | None = None,
+                 device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.device = torch.device(device)
+        self.shape = (N, Cin, Cout, H, W, k, stride, pad, dilation)
+        self.plan = mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation, opts) if opts is not None \
+            else mnn_conv_plan(N, Cin, Cout, H, W, k, stride, pad, dilation)
+        self.info = mnn_conv_plan_query(self.plan)
+        self.workspace = None
+        if self.info.workspace_bytes > 0:
+            with torch.cuda.device(self.device):
+                self.workspace = torch.empty(self.info.workspace_bytes + 1024, dtype=torch.uint8, device=self.device)
+                base = self.workspace.data_ptr()
+                self._ws_ptr = (base + 1023) // 1024 * 1024
+                mnn_conv_set_workspace(self.plan, self._ws_ptr, self.info.workspace_bytes)
+
+    def stream(self) -> int:
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def prepare(self, w) -> None:
+        mnn_conv_prepare_weights(self.plan, w.data_ptr(), self.stream())
+
+    def run(self, x, w, bias=None, y=None, stage_mask=None):
+        torch = self.torch
+        N, Cin, Cout = self.shape[0], self.shape[1], self.shape[2]
+        if y is None:
+            y = torch.empty((N, Cout, self.info.OH, self.info.OW), dtype=torch.float32, device=self.device)
+        bp = bias.data_ptr() if bias is not None else None
+        if stage_mask is None:
+            mnn_conv_run(self.plan, x.data_ptr(), w.data_ptr(), bp, y.data_ptr(), self.stream())
+        else:
+            mnn_conv_run_stages(self.plan, x.data_ptr() if x is not None else None,
+                                w.data_ptr() if w is not None else None, bp, y.data_ptr(), self.stream(), stage_mask)
+        return y
+
+    def workspace_view(self, offset: int, nbytes: int, dtype):
+        """A typed view of a workspace region (for checking the stages one by one)."""
+        torch = self.torch
+        start = self._ws_ptr - self.workspace.data_ptr() + offset
+        return self.workspace[start:start + nbytes].view(dtype)
+
+    def device_status(self) -> int:
+        return mnn_conv_device_status(self.plan, self.stream())
+
+    def close(self) -> None:
+        if self.plan:
+            mnn_conv_destroy(self.plan)
+            self.plan = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,450 @@
+// C ABI of the library: plan objects, run entry points, generator and planner access.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "../../include/mnn_conv.h"
+#include "generator.h"
+#include "kernels.h"
+#include "planner.h"
+
+using namespace mnnb;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(int code, const std::string& why)
+{
+    g_last_error = why;
+    return code;
+}
+
+int fail_cuda(cudaError_t e, const char* where)
+{
+    g_last_error = std::string(where) + ": " + cudaGetErrorString(e);
+    return MNN_ECUDA;
+}
+
+long long align_up(long long v, long long a) { return (v + a - 1) / a * a; }
+
+constexpr long long kStatusBytes = 1024;   // head of the workspace: device status word
+
+}  // namespace
+
+struct mnn_conv_plan_s {
+    LayerShape s;
+    mnn_conv_opts o;
+    Decision d;
+    int store_mode = STORE_TF32;
+    int cin_pad = 0;                 // row length of U and V (Winograd: padded Cin; GEMM: padded Cin*k*k)
+    long long chunk_tiles = 0;       // capacity of V / M in tiles (or GEMM columns)
+    int m_row_stride = 0;
+    long long u_offset = 0, u_bytes = 0, v_offset = 0, v_bytes = 0, m_offset = 0, m_bytes = 0, workspace_bytes = 0;
+    int launches_per_run = 1;
+    TransformMatrices mats;
+    // run-time state
+    char* ws = nullptr;
+    long long ws_bytes = 0;
+    const float* prepared_w = nullptr;
+    UmmaContract uc;
+};
+
+namespace {
+
+void* u_hi(mnn_conv_plan_t p) { return p->ws + p->u_offset; }
+void* u_lo(mnn_conv_plan_t p) { return store_is_split(p->store_mode) ? p->ws + p->u_offset + p->u_bytes / 2 : nullptr; }
+void* v_hi(mnn_conv_plan_t p) { return p->ws + p->v_offset; }
+void* v_lo(mnn_conv_plan_t p) { return store_is_split(p->store_mode) ? p->ws + p->v_offset + p->v_bytes / 2 : nullptr; }
+float* m_buf(mnn_conv_plan_t p) { return reinterpret_cast<float*>(p->ws + p->m_offset); }
+int* status_word(mnn_conv_plan_t p) { return reinterpret_cast<int*>(p->ws); }
+
+int store_mode_of(int operand, int passes)
+{
+    if (operand == MNN_OPERAND_FP32_REF) return STORE_FP32;
+    if (operand == MNN_OPERAND_BF16) return passes == 3 ? STORE_BF16_SPLIT : STORE_BF16;
+    return passes == 3 ? STORE_TF32_SPLIT : STORE_TF32;
+}
+
+void layout_workspace(mnn_conv_plan_t p)
+{
+    const LayerShape& s = p->s;
+    const Decision& d = p->d;
+    p->store_mode = store_mode_of(d.operand, d.passes);
+    const long long eb = store_elem_bytes(p->store_mode) * (store_is_split(p->store_mode) ? 2 : 1);
+    if (d.algo == MNN_ALGO_DIRECT) {
+        p->workspace_bytes = 0;
+        p->launches_per_run = 1;
+        return;
+    }
+    long long off = kStatusBytes;
+    if (d.algo == MNN_ALGO_WINOGRAD) {
+        const long long a2 = (long long)d.alpha * d.alpha;
+        const long long th = (s.OH + d.m - 1) / d.m, tw = (s.OW + d.m - 1) / d.m;
+        p->cin_pad = (int)align_up(s.Cin, 8);
+        p->chunk_tiles = (long long)d.chunk_images * th * tw;
+        p->m_row_stride = (int)align_up(p->chunk_tiles, 32);
+        p->u_bytes = align_up(a2 * s.Cout * p->cin_pad * eb, 2048);
+        p->v_bytes = align_up(a2 * p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->m_bytes = align_up(a2 * s.Cout * p->m_row_stride * 4, 1024);
+        p->launches_per_run = 3 * d.n_chunks;
+    } else {
+        p->cin_pad = (int)align_up((long long)s.Cin * s.k * s.k, 8);
+        p->chunk_tiles = (long long)s.N * s.OH * s.OW;
+        p->m_row_stride = 0;
+        p->u_bytes = align_up((long long)s.Cout * p->cin_pad * eb, 2048);
+        p->v_bytes = align_up(p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->m_bytes = 0;
+        p->launches_per_run = 2;
+    }
+    p->u_offset = off;
+    off += p->u_bytes;
+    p->v_offset = off;
+    off += p->v_bytes;
+    p->m_offset = off;
+    off += p->m_bytes;
+    p->workspace_bytes = off;
+}
+
+bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char* mnn_last_error(void) { return g_last_error.c_str(); }
+
+mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, int stride, int pad, int dilation,
+                                 const mnn_conv_opts* opts)
+{
+    mnn_conv_opts o;
+    std::memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    if (o.groups == 0) o.groups = 1;
+    if (N <= 0 || Cin <= 0 || Cout <= 0 || H <= 0 || W <= 0 || k <= 0 || stride <= 0 || pad < 0 || dilation <= 0) {
+        fail(MNN_EINVAL, "sizes, k, stride and dilation must be positive and pad non-negative");
+        return nullptr;
+    }
+    if (o.groups < 1 || Cin % o.groups || Cout % o.groups) {
+        fail(MNN_EINVAL, "groups must divide Cin and Cout");
+        return nullptr;
+    }
+    if (o.groups != 1 && !(o.groups == Cin && Cin == Cout)) {
+        fail(MNN_EUNSUPPORTED, "groups must be 1 or Cin = Cout (depthwise)");
+        return nullptr;
+    }
+    if (o.precision != MNN_PREC_TF32 && o.precision != MNN_PREC_BF16) {
+        fail(MNN_EINVAL, "precision must be MNN_PREC_TF32 or MNN_PREC_BF16");
+        return nullptr;
+    }
+    if (o.operand < 0 || o.operand > MNN_OPERAND_FP32_REF || !(o.passes == 0 || o.passes == 1 || o.passes == 3) ||
+        o.force_algo < 0 || o.force_algo > MNN_ALGO_DIRECT || o.points_id < 0 || o.points_id > MNN_POINTS_MIXED ||
+        o.force_m < 0 || o.chunk_images < 0) {
+        fail(MNN_EINVAL, "an option is outside its range");
+        return nullptr;
+    }
+    if (k > 11) {
+        fail(MNN_EUNSUPPORTED, "kernel sizes above 11 are not supported");
+        return nullptr;
+    }
+    LayerShape s;
+    s.N = N; s.Cin = Cin; s.Cout = Cout; s.H = H; s.W = W; s.k = k; s.stride = stride; s.pad = pad; s.dil = dilation;
+    s.groups = o.groups; s.relu = o.relu ? 1 : 0;
+    s.OH = conv_out_extent(H, k, stride, pad, dilation);
+    s.OW = conv_out_extent(W, k, stride, pad, dilation);
+    if (s.OH <= 0 || s.OW <= 0) {
+        fail(MNN_EINVAL, "the dilated kernel does not fit the padded input");
+        return nullptr;
+    }
+    if ((long long)N * Cin * H * W >= (1ll << 40) || (long long)N * Cout * s.OH * s.OW >= (1ll << 40)) {
+        fail(MNN_EUNSUPPORTED, "tensor too large");
+        return nullptr;
+    }
+    mnn_conv_plan_t p = new (std::nothrow) mnn_conv_plan_s();
+    if (!p) {
+        fail(MNN_EINVAL, "out of host memory");
+        return nullptr;
+    }
+    p->s = s;
+    p->o = o;
+    const char* why = "";
+    int rc = plan_layer(s, o, current_calibration(), &p->d, &why);
+    if (rc != MNN_OK) {
+        fail(rc, why);
+        delete p;
+        return nullptr;
+    }
+    if (p->d.algo == MNN_ALGO_WINOGRAD) {
+        WinogradMatrices wm;
+        if (!generate_winograd(p->d.m, k, p->d.points_id, &wm) || p->d.alpha > 12 || p->d.m > 6 || k > 7) {
+            fail(MNN_EUNSUPPORTED, "no transform matrices for this (m, k, points)");
+            delete p;
+            return nullptr;
+        }
+        std::memset(&p->mats, 0, sizeof(p->mats));
+        std::memcpy(p->mats.At, wm.At32.data(), wm.At32.size() * sizeof(float));
+        std::memcpy(p->mats.G, wm.G32.data(), wm.G32.size() * sizeof(float));
+        std::memcpy(p->mats.Bt, wm.Bt32.data(), wm.Bt32.size() * sizeof(float));
+    }
+    layout_workspace(p);
+    return p;
+}
+
+mnn_conv_plan_t mnn_conv_plan(int N, int Cin, int Cout, int H, int W, int k, int stride, int pad, int dilation)
+{
+    mnn_conv_opts o;
+    std::memset(&o, 0, sizeof(o));
+    o.groups = 1;
+    o.relu = 1;
+    o.precision = MNN_PREC_TF32;
+    return mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation, &o);
+}
+
+int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
+{
+    if (!p || !info) return fail(MNN_EINVAL, "NULL plan or info");
+    std::memset(info, 0, sizeof(*info));
+    info->algo = p->d.algo;
+    info->m = p->d.m;
+    info->alpha = p->d.alpha;
+    info->precision = p->o.precision;
+    info->operand = p->d.operand;
+    info->passes = p->d.passes;
+    info->points_id = p->d.points_id;
+    info->OH = p->s.OH;
+    info->OW = p->s.OW;
+    info->groups = p->s.groups;
+    info->relu = p->s.relu;
+    info->chunk_images = p->d.chunk_images;
+    info->n_chunks = p->d.n_chunks;
+    info->launches_per_run = p->launches_per_run;
+    info->cin_pad = p->cin_pad;
+    info->m_row_stride = p->m_row_stride;
+    info->chunk_tiles = p->chunk_tiles;
+    info->workspace_bytes = p->workspace_bytes;
+    info->u_offset = p->u_offset;
+    info->u_bytes = p->u_bytes;
+    info->v_offset = p->v_offset;
+    info->v_bytes = p->v_bytes;
+    info->m_offset = p->m_offset;
+    info->m_bytes = p->m_bytes;
+    info->predicted_error_ppm = p->d.error_ppm;
+    info->chosen_candidate = p->d.chosen;
+    for (int i = 0; i < MNN_N_CANDIDATES; ++i) info->cost_ps[i] = p->d.cost_ps[i];
+    return MNN_OK;
+}
+
+int mnn_conv_set_workspace(mnn_conv_plan_t p, void* workspace, long long bytes)
+{
+    if (!p) return fail(MNN_EINVAL, "NULL plan");
+    p->prepared_w = nullptr;
+    p->uc.ready = false;
+    p->ws = nullptr;
+    p->ws_bytes = 0;
+    if (p->workspace_bytes == 0) return MNN_OK;
+    if (!workspace) return fail(MNN_EWORKSPACE, "this plan needs a workspace");
+    if (bytes < p->workspace_bytes) return fail(MNN_EWORKSPACE, "workspace smaller than info.workspace_bytes");
+    if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return fail(MNN_EALIGN, "workspace must be 1024-byte aligned");
+    p->ws = static_cast<char*>(workspace);
+    p->ws_bytes = bytes;
+    cudaError_t e = cudaMemset(p->ws, 0, kStatusBytes);
+    if (e != cudaSuccess) return fail_cuda(e, "clearing the status word");
+    if (p->d.operand != MNN_OPERAND_FP32_REF) {
+        const char* why = "";
+        const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
+        e = umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p),
+                                v_hi(p), v_lo(p), &why);
+        if (e != cudaSuccess) {
+            p->ws = nullptr;
+            return fail(MNN_ECUDA, std::string("tensor-core contraction setup: ") + why + " (" + cudaGetErrorString(e) + ")");
+        }
+    }
+    return MNN_OK;
+}
+
+static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, const float* y, unsigned mask)
+{
+    if (!p) return fail(MNN_EINVAL, "NULL plan");
+    if ((mask & ~(unsigned)MNN_STAGE_ALL) || mask == 0) return fail(MNN_EINVAL, "bad stage mask");
+    if (p->workspace_bytes > 0 && !p->ws) return fail(MNN_EWORKSPACE, "call mnn_conv_set_workspace first");
+    const bool direct = p->d.algo == MNN_ALGO_DIRECT;
+    const bool need_x = direct || (mask & MNN_STAGE_INPUT);
+    const bool need_w = direct || (mask & MNN_STAGE_WEIGHT);
+    const bool need_y = direct || (mask & MNN_STAGE_OUTPUT) || (p->d.algo == MNN_ALGO_GEMM && (mask & MNN_STAGE_CONTRACT));
+    if ((need_x && !x) || (need_w && !w) || (need_y && !y)) return fail(MNN_EINVAL, "NULL tensor pointer");
+    if ((x && !aligned16(x)) || (w && !aligned16(w)) || (y && !aligned16(y)))
+        return fail(MNN_EALIGN, "x, w and y must be 16-byte aligned");
+    if (x && y && (const void*)x == (const void*)y) return fail(MNN_EINVAL, "y must not alias x");
+    return MNN_OK;
+}
+
+static int do_weights(mnn_conv_plan_t p, const float* w, cudaStream_t st)
+{
+    cudaError_t e;
+    if (p->d.algo == MNN_ALGO_WINOGRAD)
+        e = launch_weight_transform(w, u_hi(p), u_lo(p), p->s.Cout, p->s.Cin, p->s.k, p->d.m, p->cin_pad, p->store_mode,
+                                    p->mats, st);
+    else
+        e = launch_weight_round(w, u_hi(p), u_lo(p), p->s.Cout, p->s.Cin * p->s.k * p->s.k, p->cin_pad, p->store_mode, st);
+    if (e != cudaSuccess) return fail_cuda(e, "weight transform");
+    p->prepared_w = w;
+    return MNN_OK;
+}
+
+int mnn_conv_prepare_weights(mnn_conv_plan_t p, const float* w, void* stream)
+{
+    if (!p || !w) return fail(MNN_EINVAL, "NULL plan or weights");
+    if (p->d.algo == MNN_ALGO_DIRECT) {
+        p->prepared_w = w;
+        return MNN_OK;
+    }
+    if (!p->ws) return fail(MNN_EWORKSPACE, "call mnn_conv_set_workspace first");
+    if (!aligned16(w)) return fail(MNN_EALIGN, "w must be 16-byte aligned");
+    return do_weights(p, w, static_cast<cudaStream_t>(stream));
+}
+
+int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const float* bias, float* y, void* stream,
+                        unsigned mask)
+{
+    int rc = check_run_args(p, x, w, y, mask);
+    if (rc != MNN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const LayerShape& s = p->s;
+    const Decision& d = p->d;
+    cudaError_t e;
+
+    if (d.algo == MNN_ALGO_DIRECT) {
+        if (!(mask & MNN_STAGE_CONTRACT)) return MNN_OK;
+        DirectGeom g = {s.N, s.Cin, s.Cout, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, s.groups, s.relu};
+        e = launch_direct(x, w, bias, y, g, st);
+        if (e != cudaSuccess) return fail_cuda(e, "direct convolution");
+        return MNN_OK;
+    }
+
+    if (mask & MNN_STAGE_WEIGHT) {
+        rc = do_weights(p, w, st);
+        if (rc != MNN_OK) return rc;
+    }
+    const bool reference = d.operand == MNN_OPERAND_FP32_REF;
+
+    if (d.algo == MNN_ALGO_GEMM) {
+        const long long T = (long long)s.N * s.OH * s.OW;
+        if (mask & MNN_STAGE_INPUT) {
+            GatherGeom g = {s.N, s.Cin, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, p->cin_pad};
+            e = launch_gather(x, v_hi(p), v_lo(p), g, p->store_mode, st);
+            if (e != cudaSuccess) return fail_cuda(e, "patch gather");
+        }
+        if (mask & MNN_STAGE_CONTRACT) {
+            ContractEpilogue epi = {1, nullptr, 0, y, bias, s.relu, s.OH * s.OW};
+            if (reference)
+                e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, 1, s.Cout, T, p->cin_pad,
+                                              (long long)s.Cout * p->cin_pad, T * p->cin_pad, epi, st);
+            else
+                e = launch_contract_umma(p->uc, T, epi, status_word(p), st);
+            if (e != cudaSuccess) return fail_cuda(e, "GEMM contraction");
+        }
+        return MNN_OK;
+    }
+
+    // Winograd: the three stages chunk by chunk, so that one chunk's V and M stay in L2.
+    const int th = (s.OH + d.m - 1) / d.m, tw = (s.OW + d.m - 1) / d.m;
+    const int alpha2 = d.alpha * d.alpha;
+    for (int n0 = 0; n0 < s.N; n0 += d.chunk_images) {
+        const int n_img = (s.N - n0) < d.chunk_images ? (s.N - n0) : d.chunk_images;
+        WinoGeom g;
+        g.images = n_img;
+        g.Cin = s.Cin; g.Cout = s.Cout; g.H = s.H; g.W = s.W; g.OH = s.OH; g.OW = s.OW; g.k = s.k; g.pad = s.pad;
+        g.m = d.m; g.alpha = d.alpha; g.th = th; g.tw = tw; g.cin_pad = p->cin_pad;
+        g.tiles = (long long)n_img * th * tw;
+        g.v_plane = p->chunk_tiles * p->cin_pad;
+        g.m_row_stride = p->m_row_stride;
+        if (mask & MNN_STAGE_INPUT) {
+            e = launch_input_transform(x + (size_t)n0 * s.Cin * s.H * s.W, v_hi(p), v_lo(p), g, p->store_mode, p->mats, st);
+            if (e != cudaSuccess) return fail_cuda(e, "input transform");
+        }
+        if (mask & MNN_STAGE_CONTRACT) {
+            ContractEpilogue epi = {0, m_buf(p), p->m_row_stride, nullptr, nullptr, 0, 1};
+            if (reference)
+                e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, alpha2, s.Cout, g.tiles,
+                                              p->cin_pad, (long long)s.Cout * p->cin_pad, g.v_plane, epi, st);
+            else
+                e = launch_contract_umma(p->uc, g.tiles, epi, status_word(p), st);
+            if (e != cudaSuccess) return fail_cuda(e, "Winograd contraction");
+        }
+        if (mask & MNN_STAGE_OUTPUT) {
+            e = launch_output_transform(m_buf(p), bias, y + (size_t)n0 * s.Cout * s.OH * s.OW, g, s.relu, p->mats, st);
+            if (e != cudaSuccess) return fail_cuda(e, "output transform");
+        }
+    }
+    return MNN_OK;
+}
+
+int mnn_conv_run(mnn_conv_plan_t p, const float* x, const float* w, const float* bias, float* y, void* stream)
+{
+    if (!p) return fail(MNN_EINVAL, "NULL plan");
+    if (!x || !w || !y) return fail(MNN_EINVAL, "NULL tensor pointer");
+    unsigned mask = MNN_STAGE_INPUT | MNN_STAGE_CONTRACT | MNN_STAGE_OUTPUT;
+    if (p->d.algo != MNN_ALGO_DIRECT && p->prepared_w != w) mask |= MNN_STAGE_WEIGHT;
+    return mnn_conv_run_stages(p, x, w, bias, y, stream, mask);
+}
+
+int mnn_conv_device_status(mnn_conv_plan_t p, void* stream, int* code)
+{
+    if (!p || !code) return fail(MNN_EINVAL, "NULL plan or code");
+    *code = 0;
+    if (!p->ws) return MNN_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(code, status_word(p), sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail_cuda(e, "reading the status word");
+    if (*code != 0) {
+        e = cudaMemsetAsync(status_word(p), 0, sizeof(int), st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return fail_cuda(e, "clearing the status word");
+    }
+    return MNN_OK;
+}
+
+void mnn_conv_destroy(mnn_conv_plan_t p) { delete p; }
+
+int mnn_winograd_matrices(int m, int k, int points_id, float* At, float* G, float* Bt)
+{
+    WinogradMatrices wm;
+    if (points_id < 1 || points_id > 3) return fail(MNN_EINVAL, "points_id must be 1, 2 or 3");
+    if (!generate_winograd(m, k, points_id, &wm)) return fail(MNN_EINVAL, "need m, k >= 1 and m + k - 1 <= 16 within the point set");
+    if (At) std::memcpy(At, wm.At32.data(), wm.At32.size() * sizeof(float));
+    if (G) std::memcpy(G, wm.G32.data(), wm.G32.size() * sizeof(float));
+    if (Bt) std::memcpy(Bt, wm.Bt32.data(), wm.Bt32.size() * sizeof(float));
+    return MNN_OK;
+}
+
+long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int passes)
+{
+    long long v = accuracy_ppm(m, k, points_id, operand, passes);
+    if (v < 0) fail(MNN_EINVAL, "invalid (m, k, points_id, operand, passes)");
+    return v;
+}
+
+int mnn_set_calibration(const long long consts[MNN_N_CONSTS])
+{
+    if (!consts) return fail(MNN_EINVAL, "NULL constants");
+    Calibration c;
+    for (int i = 0; i < MNN_N_CONSTS; ++i) c.c[i] = consts[i];
+    for (int i = 0; i <= 8; ++i)
+        if (c.c[i] <= 0) return fail(MNN_EINVAL, "constants 0..8 must be positive");
+    install_calibration(c);
+    return MNN_OK;
+}
+
+int mnn_get_calibration(long long consts[MNN_N_CONSTS])
+{
+    if (!consts) return fail(MNN_EINVAL, "NULL constants");
+    Calibration c = current_calibration();
+    for (int i = 0; i < MNN_N_CONSTS; ++i) consts[i] = c.c[i];
+    return MNN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,376 @@
+// Batched channel contraction on the 5th-generation tensor cores (Section 3.3.1 (2):
+// the Hadamard product of Eq. 6 summed over channels, recast as one matrix product
+// per transform position xi):
+//     out[xi][co][t] = sum_c V[xi][t][c] * U[xi][co][c]
+// A persistent, warp-specialised kernel: one thread feeds shared memory with TMA
+// (128-byte-swizzled K-major tiles of V and U), one thread issues tcgen05.mma with
+// the accumulator in tensor memory (128 tiles x BN output channels, double
+// buffered), four warps drain the accumulator with tcgen05.ld and store it.
+// The MMA "M" dimension is the tile index t, "N" the output channel, "K" the input
+// channel; TF32 or BF16 operands, fp32 accumulation; with passes = 3 the operands
+// come as hi + lo pairs and hi*hi + lo*hi + hi*lo are accumulated.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+#include "umma.cuh"
+
+namespace mnnb {
+
+namespace {
+
+constexpr int kThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kTileM = 128;            // tiles (rows of V) per work item
+constexpr int kMaxStages = 8;
+constexpr int kSwizzleBytes = 128;     // bytes of K per shared-memory row
+constexpr int kSmemBudget = 200 * 1024;
+
+struct KernelParams {
+    int alpha2, n_tile_blocks, n_co_blocks, bn, k_blocks, passes, stages, tmem_cols;
+    int Cout;
+    long long tiles;
+    long long n_items;
+    ContractEpilogue epi;
+    int* status;
+};
+
+// status codes written on a bounded wait that ran out
+constexpr int kErrProducerWait = 1, kErrMmaWaitFull = 2, kErrMmaWaitTmem = 3, kErrEpilogueWait = 4;
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_constant__ CUtensorMap map_v_lo,
+                     const __grid_constant__ CUtensorMap map_u_hi, const __grid_constant__ CUtensorMap map_u_lo,
+                     KernelParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t tfull_bar[2];
+    __shared__ __align__(8) uint64_t tempty_bar[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_bytes = kTileM * kSwizzleBytes;                 // one V tile
+    const uint32_t b_bytes = (uint32_t)p.bn * kSwizzleBytes;         // one U tile
+    const uint32_t split = p.passes == 3 ? 2u : 1u;
+    const uint32_t stage_bytes = (a_bytes + b_bytes) * split;
+    // stage layout: [A_hi][A_lo?][B_hi][B_lo?]
+    const uint32_t off_a_lo = a_bytes, off_b_hi = a_bytes * split, off_b_lo = a_bytes * split + b_bytes;
+    volatile int* abortp = &abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&full_bar[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&empty_bar[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&tfull_bar[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&tempty_bar[s]), 128);
+        }
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&map_v_hi);
+        ptx::prefetch_tensormap(&map_u_hi);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), (uint32_t)p.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+
+    const int k_elems = KIND == 0 ? 32 : 64;         // elements of K per 128-byte row
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (long long item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+                const int tb = (int)(item % p.n_tile_blocks);
+                const long long r = item / p.n_tile_blocks;
+                const int nb = (int)(r % p.n_co_blocks);
+                const int xi = (int)(r / p.n_co_blocks);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, abortp)) {
+                        if (!*abortp) atomicCAS(p.status, 0, kErrProducerWait);
+                        *abortp = 1;
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
+                    const uint32_t sbase = smem_base + stage * stage_bytes;
+                    ptx::mbar_expect_tx(bar, stage_bytes);
+                    ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
+                    ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
+                    if (split == 2) {
+                        ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM, xi);
+                        ptx::tma_load_3d(sbase + off_b_lo, &map_u_lo, bar, kb * k_elems, nb * p.bn, xi);
+                    }
+                    if (++stage == (uint32_t)p.stages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = ptx::mma_idesc(KIND == 0 ? 2 : 1, kTileM, p.bn);
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (long long item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, abortp)) {
+                    if (!*abortp) atomicCAS(p.status, 0, kErrMmaWaitTmem);
+                    *abortp = 1;
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.bn;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full_bar[stage]), phase, abortp)) {
+                        if (!*abortp) atomicCAS(p.status, 0, kErrMmaWaitFull);
+                        *abortp = 1;
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t sbase = smem_base + stage * stage_bytes;
+#pragma unroll
+                    for (int ks = 0; ks < kSwizzleBytes / 32; ++ks) {
+                        const uint64_t a_hi = ptx::smem_desc_k128(sbase + ks * 32);
+                        const uint64_t b_hi = ptx::smem_desc_k128(sbase + off_b_hi + ks * 32);
+                        ptx::mma_ss<KIND>(d_tmem, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
+                        if (split == 2) {
+                            const uint64_t a_lo = ptx::smem_desc_k128(sbase + off_a_lo + ks * 32);
+                            const uint64_t b_lo = ptx::smem_desc_k128(sbase + off_b_lo + ks * 32);
+                            ptx::mma_ss<KIND>(d_tmem, a_lo, b_hi, idesc, 1u);
+                            ptx::mma_ss<KIND>(d_tmem, a_hi, b_lo, idesc, 1u);
+                        }
+                    }
+                    ptx::mma_commit(ptx::smem_u32(&empty_bar[stage]));     // stage reusable once these MMAs retire
+                    if (++stage == (uint32_t)p.stages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                ptx::mma_commit(ptx::smem_u32(&tfull_bar[acc]));           // accumulator complete
+                acc ^= 1u;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+        }
+    } else {
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (long long item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+            const int tb = (int)(item % p.n_tile_blocks);
+            const long long r = item / p.n_tile_blocks;
+            const int nb = (int)(r % p.n_co_blocks);
+            const int xi = (int)(r / p.n_co_blocks);
+            if (!ptx::mbar_wait_bounded(ptx::smem_u32(&tfull_bar[acc]), acc_phase, abortp)) {
+                if (!*abortp) atomicCAS(p.status, 0, kErrEpilogueWait);
+                *abortp = 1;
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after();
+            const long long t = (long long)tb * kTileM + q * 32 + lane;
+            const bool t_ok = t < p.tiles;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)p.bn;
+            float* out_row = nullptr;
+            long long img = 0, pix = 0;
+            if (p.epi.mode == 0) {
+                out_row = p.epi.M + (size_t)xi * p.Cout * p.epi.m_row_stride + t;
+            } else {
+                img = t / p.epi.ohw;
+                pix = t % p.epi.ohw;
+            }
+            for (int c0 = 0; c0 < p.bn; c0 += 16) {
+                uint32_t v[16];
+                ptx::tmem_ld16(taddr + (uint32_t)c0, v);
+                ptx::tmem_ld_wait();
+                const int co_base = nb * p.bn + c0;
+                if (t_ok) {
+                    if (p.epi.mode == 0) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int co = co_base + j;
+                            if (co < p.Cout) out_row[(size_t)co * p.epi.m_row_stride] = __uint_as_float(v[j]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int co = co_base + j;
+                            if (co < p.Cout) {
+                                float s = __uint_as_float(v[j]) + (p.epi.bias ? __ldg(p.epi.bias + co) : 0.0f);
+                                if (p.epi.relu) s = fmaxf(s, 0.0f);
+                                p.epi.y[((size_t)img * p.Cout + co) * p.epi.ohw + pix] = s;
+                            }
+                        }
+                    }
+                }
+            }
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(ptx::smem_u32(&tempty_bar[acc]));
+            acc ^= 1u;
+            if (acc == 0) acc_phase ^= 1u;
+        }
+    }
+
+    // Teardown.  After an aborted run give copies still in flight time to land before the CTA's
+    // shared memory is released.
+    if (*abortp) __nanosleep(200000);
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// 3-D map over [planes][rows][k] (k contiguous), box = [1][box_rows][128 bytes of k], 128-byte swizzle.
+bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
+                        long long plane_stride_elems, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)k_len, (cuuint64_t)rows, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)k_len * elem_bytes, (cuuint64_t)plane_stride_elems * elem_bytes};
+    const cuuint32_t box[3] = {(cuuint32_t)(kSwizzleBytes / elem_bytes), (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    CUresult r = fn(map, dt, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout, int cin_pad, long long tiles_capacity,
+                                void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why)
+{
+    uc->ready = false;
+    if (mode == STORE_FP32) {
+        *why = "the tensor-core contraction needs TF32 or BF16 operands";
+        return cudaErrorInvalidValue;
+    }
+    const int eb = store_elem_bytes(mode);
+    uc->kind = eb == 2 ? 1 : 0;
+    uc->passes = store_is_split(mode) ? 3 : 1;
+    uc->alpha2 = alpha2;
+    uc->Cout = Cout;
+    uc->cin_pad = cin_pad;
+    uc->tiles_capacity = tiles_capacity;
+    if (((long long)cin_pad * eb) % 16 != 0) {
+        *why = "operand rows must be a multiple of 16 bytes";
+        return cudaErrorInvalidValue;
+    }
+    // output channels per MMA: as many as fit (<= 256), multiple of 16, blocks balanced
+    const int co16 = (Cout + 15) / 16 * 16;
+    uc->n_co_blocks = (co16 + 255) / 256;
+    uc->bn = ((co16 / 16 + uc->n_co_blocks - 1) / uc->n_co_blocks) * 16;
+    const int k_elems = kSwizzleBytes / eb;
+    uc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
+    const int split = uc->passes == 3 ? 2 : 1;
+    const int stage_bytes = (kTileM * kSwizzleBytes + uc->bn * kSwizzleBytes) * split;
+    int stages = (kSmemBudget - 1024) / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) {
+        *why = "shared memory cannot hold two pipeline stages";
+        return cudaErrorInvalidValue;
+    }
+    uc->stages = stages;
+    // Always ask for the full budget so that at most one CTA is resident per SM: a second CTA could
+    // otherwise block inside the tensor-memory allocation.
+    uc->smem_bytes = kSmemBudget;
+    int cols = 32;
+    while (cols < 2 * uc->bn) cols *= 2;
+    uc->tmem_cols = cols;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&uc->num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+
+    const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
+    bool ok = encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
+              encode_operand_map(&uc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
+    if (ok && split == 2)
+        ok = encode_operand_map(&uc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
+             encode_operand_map(&uc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
+    if (!ok) {
+        *why = "cuTensorMapEncodeTiled failed or is unavailable";
+        return cudaErrorInvalidValue;
+    }
+    if (split == 1) {
+        uc->map_v_lo = uc->map_v_hi;
+        uc->map_u_lo = uc->map_u_hi;
+    }
+    auto k0 = contract_umma_kernel<0>;
+    auto k1 = contract_umma_kernel<1>;
+    e = cudaFuncSetAttribute(k0, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return e;
+    uc->ready = true;
+    return cudaSuccess;
+}
+
+cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const ContractEpilogue& epi, int* status,
+                                 cudaStream_t stream)
+{
+    if (!uc.ready) return cudaErrorInvalidValue;
+    if (tiles <= 0) return cudaSuccess;
+    if (tiles > uc.tiles_capacity) return cudaErrorInvalidValue;
+    KernelParams p;
+    p.alpha2 = uc.alpha2;
+    p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
+    p.n_co_blocks = uc.n_co_blocks;
+    p.bn = uc.bn;
+    p.k_blocks = uc.k_blocks;
+    p.passes = uc.passes;
+    p.stages = uc.stages;
+    p.tmem_cols = uc.tmem_cols;
+    p.Cout = uc.Cout;
+    p.tiles = tiles;
+    p.n_items = (long long)p.n_tile_blocks * p.n_co_blocks * uc.alpha2;
+    p.epi = epi;
+    p.status = status;
+    long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
+    if (uc.kind == 0)
+        contract_umma_kernel<0><<<(unsigned)grid, kThreads, uc.smem_bytes, stream>>>(uc.map_v_hi, uc.map_v_lo, uc.map_u_hi,
+                                                                                     uc.map_u_lo, p);
+    else
+        contract_umma_kernel<1><<<(unsigned)grid, kThreads, uc.smem_bytes, stream>>>(uc.map_v_hi, uc.map_v_lo, uc.map_u_hi,
+                                                                                     uc.map_u_lo, p);
+    return cudaGetLastError();
+}
+
+}  // namespace mnnb

@@ -1,0 +1,506 @@
+// Pre-inference planner (Section 3.2): choose the computation scheme of one
+// convolution layer by minimising a cost, Eq. 1.  The paper's arithmetic count
+// (Eq. 2) and its backend term MUL/FLOPS + t_schedule (Eq. 5) are re-stated for a
+// GPU whose kernels are bound by memory traffic, tensor throughput or ALU
+// throughput, whichever is largest:
+//     cost(candidate) = sum over its kernels of
+//         max(bytes x c_byte, tensor flops x c_tensor, ALU flops x c_alu) / 1e6 + c_launch
+// in integer picoseconds (the constants are attoseconds per unit).  Everything
+// below the accuracy model is integer arithmetic, so that a choice can be
+// reproduced bit for bit from the nine layer integers and the constant record.
+#include "planner.h"
+
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <vector>
+
+#include "generator.h"
+
+namespace mnnb {
+
+namespace {
+std::mutex g_cal_mutex;
+Calibration g_cal;
+bool g_cal_set = false;
+
+uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+uint64_t round_up(uint64_t a, uint64_t b) { return ceil_div(a, b) * b; }
+uint64_t max3(uint64_t a, uint64_t b, uint64_t c) { return a > b ? (a > c ? a : c) : (b > c ? b : c); }
+}  // namespace
+
+Calibration default_calibration()
+{
+    Calibration c;
+    std::memset(&c, 0, sizeof(c));
+    c.c[0] = 160000;      // as per HBM byte          (~6.2 TB/s)
+    c.c[1] = 70000;       // as per L2-resident byte  (~14 TB/s)
+    c.c[2] = 2000;        // as per TF32 tensor flop  (~500 TFLOP/s achieved)
+    c.c[3] = 1000;        // as per BF16 tensor flop  (~1000 TFLOP/s achieved)
+    c.c[4] = 28000;       // as per fp32 ALU flop in the transform kernels (~36 TFLOP/s)
+    c.c[5] = 2500000;     // ps per kernel launch (the t_schedule of Eq. 5)
+    c.c[6] = 80ll << 20;  // L2 bytes one chunk's V + M may occupy
+    c.c[7] = 148;         // SMs
+    c.c[8] = 100000;      // as per flop of the direct kernel (~10 TFLOP/s)
+    return c;
+}
+
+Calibration current_calibration()
+{
+    std::lock_guard<std::mutex> lk(g_cal_mutex);
+    return g_cal_set ? g_cal : default_calibration();
+}
+
+void install_calibration(const Calibration& c)
+{
+    std::lock_guard<std::mutex> lk(g_cal_mutex);
+    g_cal = c;
+    g_cal_set = true;
+}
+
+int conv_out_extent(int in, int k, int stride, int pad, int dil)
+{
+    if (stride <= 0) return 0;
+    long long span = (long long)in + 2ll * pad - (long long)dil * (k - 1) - 1;
+    if (span < 0) return 0;
+    return (int)(span / stride) + 1;
+}
+
+bool winograd_supported(int m, int k)
+{
+    if (!(m == 2 || m == 4 || m == 6)) return false;
+    if (!(k == 2 || k == 3 || k == 5 || k == 7)) return false;
+    return m + k - 1 <= 12;
+}
+
+// ---------------------------------------------------------------------------
+// Accuracy model: simulate F(m,k) on a fixed pseudo-random problem in fp64 with
+// U and V rounded to the operand format (optionally split into hi + lo), and
+// report the relative L2 error against the plain correlation.
+// ---------------------------------------------------------------------------
+namespace {
+
+struct Lcg {
+    uint64_t s;
+    explicit Lcg(uint64_t seed) : s(seed) {}
+    double uniform()
+    {
+        s = s * 6364136223846793005ull + 1442695040888963407ull;
+        return (double)(s >> 11) * (1.0 / 9007199254740992.0);
+    }
+    // sum of twelve uniforms minus six: mean 0, variance 1, additions only
+    double normalish()
+    {
+        double a = 0.0;
+        for (int i = 0; i < 12; ++i) a += uniform();
+        return a - 6.0;
+    }
+};
+
+double round_mantissa(double v, int bits)
+{
+    // nearest-even rounding of fp32(v) to `bits` explicit mantissa bits
+    float f = (float)v;
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    const int drop = 23 - bits;
+    if (drop > 0) {
+        uint32_t lsb = (u >> drop) & 1u;
+        u += (1u << (drop - 1)) - 1u + lsb;
+        u &= ~((1u << drop) - 1u);
+    }
+    std::memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+void split_operand(double v, int bits, int passes, double* hi, double* lo)
+{
+    *hi = round_mantissa(v, bits);
+    *lo = passes == 3 ? round_mantissa((double)(float)v - *hi, bits) : 0.0;
+}
+
+std::mutex g_acc_mutex;
+std::map<std::tuple<int, int, int, int, int>, long long> g_acc_cache;
+
+long long simulate_ppm(int m, int k, int points_id, int bits, int passes)
+{
+    const int C = 64, CO = 4, TILES = 16;
+    Lcg rng(0x9E3779B97F4A7C15ull ^ (uint64_t)(m * 1000 + k * 10));   // same data for every point set
+    const bool gemm = (m == 1 && points_id == 0);
+    WinogradMatrices wm;
+    if (!gemm && !generate_winograd(m, k, points_id, &wm)) return -1;
+    const int alpha = m + k - 1;
+    const int a2 = alpha * alpha;
+
+    std::vector<double> w((size_t)CO * C * k * k), x((size_t)TILES * C * a2);
+    const double wscale = 1.0 / std::sqrt((double)(C * k * k));
+    for (auto& v : w) v = (double)(float)(rng.normalish() * wscale);
+    for (auto& v : x) v = (double)(float)rng.normalish();
+
+    double num = 0.0, den = 0.0;
+    if (gemm) {
+        // one dot product of length C*k*k per output, operands rounded directly
+        for (int t = 0; t < TILES; ++t)
+            for (int co = 0; co < CO; ++co) {
+                double ref = 0.0, got = 0.0;
+                for (int c = 0; c < C; ++c)
+                    for (int e = 0; e < k * k; ++e) {
+                        const double wv = w[((size_t)co * C + c) * k * k + e];
+                        const double xv = x[((size_t)t * C + c) * a2 + e];
+                        double wh, wl, xh, xl;
+                        split_operand(wv, bits, passes, &wh, &wl);
+                        split_operand(xv, bits, passes, &xh, &xl);
+                        ref += wv * xv;
+                        got += wh * xh + wl * xh + wh * xl;
+                    }
+                num += (got - ref) * (got - ref);
+                den += ref * ref;
+            }
+    } else {
+        const std::vector<double>&G = wm.G64, &Bt = wm.Bt64, &At = wm.At64;
+        // U hi/lo [co][c][a2], V hi/lo [t][c][a2]
+        std::vector<double> Uh((size_t)CO * C * a2), Ul(Uh.size()), Vh((size_t)TILES * C * a2), Vl(Vh.size());
+        std::vector<double> tmp((size_t)alpha * alpha);
+        for (int co = 0; co < CO; ++co)
+            for (int c = 0; c < C; ++c) {
+                const double* g = &w[((size_t)co * C + c) * k * k];
+                for (int i = 0; i < alpha; ++i)
+                    for (int b = 0; b < k; ++b) {
+                        double s = 0.0;
+                        for (int a = 0; a < k; ++a) s += G[i * k + a] * g[a * k + b];
+                        tmp[i * k + b] = s;
+                    }
+                for (int i = 0; i < alpha; ++i)
+                    for (int j = 0; j < alpha; ++j) {
+                        double s = 0.0;
+                        for (int b = 0; b < k; ++b) s += tmp[i * k + b] * G[j * k + b];
+                        split_operand(s, bits, passes, &Uh[((size_t)co * C + c) * a2 + i * alpha + j],
+                                      &Ul[((size_t)co * C + c) * a2 + i * alpha + j]);
+                    }
+            }
+        for (int t = 0; t < TILES; ++t)
+            for (int c = 0; c < C; ++c) {
+                const double* d = &x[((size_t)t * C + c) * a2];
+                for (int i = 0; i < alpha; ++i)
+                    for (int b = 0; b < alpha; ++b) {
+                        double s = 0.0;
+                        for (int a = 0; a < alpha; ++a) s += Bt[i * alpha + a] * d[a * alpha + b];
+                        tmp[i * alpha + b] = s;
+                    }
+                for (int i = 0; i < alpha; ++i)
+                    for (int j = 0; j < alpha; ++j) {
+                        double s = 0.0;
+                        for (int b = 0; b < alpha; ++b) s += tmp[i * alpha + b] * Bt[j * alpha + b];
+                        split_operand(s, bits, passes, &Vh[((size_t)t * C + c) * a2 + i * alpha + j],
+                                      &Vl[((size_t)t * C + c) * a2 + i * alpha + j]);
+                    }
+            }
+        std::vector<double> Mx((size_t)a2), t2((size_t)m * alpha);
+        for (int t = 0; t < TILES; ++t)
+            for (int co = 0; co < CO; ++co) {
+                for (int e = 0; e < a2; ++e) {
+                    double s = 0.0;
+                    for (int c = 0; c < C; ++c) {
+                        const size_t ui = ((size_t)co * C + c) * a2 + e, vi = ((size_t)t * C + c) * a2 + e;
+                        s += Uh[ui] * Vh[vi] + Ul[ui] * Vh[vi] + Uh[ui] * Vl[vi];
+                    }
+                    Mx[e] = (double)(float)s;
+                }
+                for (int a = 0; a < m; ++a)
+                    for (int j = 0; j < alpha; ++j) {
+                        double s = 0.0;
+                        for (int i = 0; i < alpha; ++i) s += At[a * alpha + i] * Mx[i * alpha + j];
+                        t2[a * alpha + j] = s;
+                    }
+                for (int a = 0; a < m; ++a)
+                    for (int b = 0; b < m; ++b) {
+                        double got = 0.0;
+                        for (int j = 0; j < alpha; ++j) got += t2[a * alpha + j] * At[b * alpha + j];
+                        double ref = 0.0;
+                        for (int c = 0; c < C; ++c)
+                            for (int i = 0; i < k; ++i)
+                                for (int j = 0; j < k; ++j)
+                                    ref += w[((size_t)co * C + c) * k * k + i * k + j] *
+                                           x[((size_t)t * C + c) * a2 + (a + i) * alpha + (b + j)];
+                        num += (got - ref) * (got - ref);
+                        den += ref * ref;
+                    }
+            }
+    }
+    if (!(den > 0.0)) return -1;
+    const double rel = std::sqrt(num / den);
+    double ppm = std::ceil(rel * 1e6);
+    if (ppm > 4e18) ppm = 4e18;
+    return (long long)ppm;
+}
+
+}  // namespace
+
+long long accuracy_ppm(int m, int k, int points_id, int operand, int passes)
+{
+    if (m < 1 || k < 1 || m + k - 1 > kMaxAlpha) return -1;
+    if (!(operand == MNN_OPERAND_TF32 || operand == MNN_OPERAND_BF16 || operand == MNN_OPERAND_FP32_REF)) return -1;
+    if (!(passes == 1 || passes == 3)) return -1;
+    const bool gemm = (m == 1 && points_id == 0);
+    if (!gemm && (points_id < 1 || points_id > 3)) return -1;
+    const int bits = operand == MNN_OPERAND_TF32 ? 10 : (operand == MNN_OPERAND_BF16 ? 7 : 23);
+    auto key = std::make_tuple(m, k, points_id, bits, passes);
+    {
+        std::lock_guard<std::mutex> lk(g_acc_mutex);
+        auto it = g_acc_cache.find(key);
+        if (it != g_acc_cache.end()) return it->second;
+    }
+    long long v = simulate_ppm(m, k, points_id, bits, passes);
+    std::lock_guard<std::mutex> lk(g_acc_mutex);
+    g_acc_cache[key] = v;
+    return v;
+}
+
+int best_points(int m, int k, int operand, int passes, long long* ppm_out)
+{
+    int best = 0;
+    long long best_ppm = -1;
+    for (int pid = 1; pid <= 3; ++pid) {
+        long long p = accuracy_ppm(m, k, pid, operand, passes);
+        if (p < 0) continue;
+        if (best == 0 || p < best_ppm) {
+            best = pid;
+            best_ppm = p;
+        }
+    }
+    if (ppm_out) *ppm_out = best_ppm;
+    return best;
+}
+
+// ---------------------------------------------------------------------------
+// Cost model (integers only).
+// ---------------------------------------------------------------------------
+namespace {
+
+uint64_t kernel_ps(uint64_t as_mem, uint64_t as_tensor, uint64_t as_alu, const Calibration& cal)
+{
+    return max3(as_mem, as_tensor, as_alu) / 1000000ull + (uint64_t)cal.c[5];
+}
+
+uint64_t operand_bytes(int operand) { return operand == MNN_OPERAND_BF16 ? 2 : 4; }
+uint64_t tensor_as(int operand, const Calibration& cal) { return (uint64_t)(operand == MNN_OPERAND_BF16 ? cal.c[3] : cal.c[2]); }
+
+uint64_t direct_cost(const LayerShape& s, const Calibration& cal)
+{
+    const uint64_t x_bytes = 4ull * s.N * s.Cin * s.H * s.W;
+    const uint64_t y_bytes = 4ull * s.N * s.Cout * s.OH * s.OW;
+    const uint64_t w_bytes = 4ull * s.Cout * (s.Cin / s.groups) * s.k * s.k;
+    const uint64_t flops = 2ull * s.N * s.Cout * (s.Cin / s.groups) * s.OH * s.OW * s.k * s.k;
+    return kernel_ps((x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, flops * (uint64_t)cal.c[8], cal);
+}
+
+uint64_t gemm_cost(const LayerShape& s, int operand, const Calibration& cal)
+{
+    const uint64_t b = operand_bytes(operand);
+    const uint64_t Kp = round_up((uint64_t)s.Cin * s.k * s.k, 8);
+    const uint64_t T = (uint64_t)s.N * s.OH * s.OW;
+    const uint64_t x_bytes = 4ull * s.N * s.Cin * s.H * s.W;
+    const uint64_t y_bytes = 4ull * s.N * s.Cout * s.OH * s.OW;
+    const uint64_t v_bytes = T * Kp * b, u_bytes = (uint64_t)s.Cout * Kp * b;
+    const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0], 0, 0, cal);
+    const uint64_t contract = kernel_ps((v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0],
+                                        2ull * T * s.Cout * Kp * tensor_as(operand, cal), 0, cal);
+    return gather + contract;
+}
+
+uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes, uint64_t n, bool resident,
+                             const Calibration& cal)
+{
+    const uint64_t alpha = (uint64_t)(m + s.k - 1), a2 = alpha * alpha;
+    const uint64_t tiles_img = ceil_div(s.OH, m) * ceil_div(s.OW, m);
+    const uint64_t Cp = round_up(s.Cin, 8);
+    const uint64_t b_el = operand_bytes(operand) * (passes == 3 ? 2 : 1);
+    const uint64_t v_bytes = n * a2 * tiles_img * Cp * b_el;
+    const uint64_t m_bytes = n * a2 * (uint64_t)s.Cout * tiles_img * 4;
+    const uint64_t u_bytes = a2 * (uint64_t)s.Cout * Cp * b_el;
+    const uint64_t x_bytes = 4ull * n * s.Cin * s.H * s.W;
+    const uint64_t y_bytes = 4ull * n * s.Cout * s.OH * s.OW;
+    const uint64_t cV = (uint64_t)(resident ? cal.c[1] : cal.c[0]);
+    const uint64_t c0 = (uint64_t)cal.c[0], cA = (uint64_t)cal.c[4];
+    const uint64_t in = kernel_ps(x_bytes * c0 + v_bytes * cV, 0, 4ull * alpha * a2 * n * tiles_img * s.Cin * cA, cal);
+    const uint64_t con = kernel_ps((v_bytes + m_bytes) * cV + u_bytes * c0,
+                                   2ull * a2 * s.Cout * Cp * n * tiles_img * passes * tensor_as(operand, cal), 0, cal);
+    const uint64_t out = kernel_ps(m_bytes * cV + y_bytes * c0, 0,
+                                   2ull * m * alpha * (alpha + m) * n * tiles_img * s.Cout * cA, cal);
+    return in + con + out;
+}
+
+}  // namespace
+
+void winograd_chunking(const LayerShape& s, int m, int operand, int passes, const Calibration& cal,
+                       int* chunk_images, int* n_chunks, uint64_t* cost_ps)
+{
+    const uint64_t alpha = (uint64_t)(m + s.k - 1), a2 = alpha * alpha;
+    const uint64_t tiles_img = ceil_div(s.OH, m) * ceil_div(s.OW, m);
+    const uint64_t Cp = round_up(s.Cin, 8);
+    const uint64_t b_el = operand_bytes(operand) * (passes == 3 ? 2 : 1);
+    const uint64_t per_img = a2 * tiles_img * Cp * b_el + a2 * (uint64_t)s.Cout * tiles_img * 4;
+    const uint64_t N = (uint64_t)s.N;
+    const uint64_t n_fit = per_img ? (uint64_t)cal.c[6] / per_img : N;
+
+    // option A: the whole batch in one chunk
+    const uint64_t costA = winograd_chunk_cost(s, m, operand, passes, N, n_fit >= N, cal);
+    uint64_t best_cost = costA;
+    uint64_t best_chunk = N, best_n = 1;
+    if (n_fit >= 1 && n_fit < N) {
+        // option B: chunks whose V + M stay in L2
+        const uint64_t nch = ceil_div(N, n_fit);
+        const uint64_t chunk = ceil_div(N, nch);
+        const uint64_t costB = nch * winograd_chunk_cost(s, m, operand, passes, chunk, true, cal);
+        if (costB <= costA) {
+            best_cost = costB;
+            best_chunk = chunk;
+            best_n = ceil_div(N, chunk);
+        }
+    }
+    *chunk_images = (int)best_chunk;
+    *n_chunks = (int)best_n;
+    *cost_ps = best_cost;
+}
+
+int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& cal, Decision* d, const char** err)
+{
+    static const int kM[3] = {2, 4, 6};
+    for (int i = 0; i < MNN_N_CANDIDATES; ++i) d->cost_ps[i] = MNN_COST_INADMISSIBLE;
+
+    const uint64_t tol_ppm = o.precision == MNN_PREC_BF16 ? 10000 : 1000;
+    const uint64_t gate_ppm = tol_ppm * kGateNumerator / kGateDenominator;
+    const bool fully_forced = o.force_m != 0 && o.operand != 0 && o.passes != 0;
+    const bool wino_shape_ok = s.stride == 1 && s.dil == 1 && s.groups == 1 && s.k >= 2 && s.k <= 7;
+
+    struct Cand { int algo, m, operand, passes; };
+    Cand cands[MNN_N_CANDIDATES];
+    cands[0] = {MNN_ALGO_DIRECT, 0, 0, 0};
+    cands[1] = {MNN_ALGO_GEMM, 0, MNN_OPERAND_TF32, 1};
+    cands[2] = {MNN_ALGO_GEMM, 0, MNN_OPERAND_BF16, 1};
+    for (int g = 0; g < 4; ++g)
+        for (int i = 0; i < 3; ++i)
+            cands[3 + g * 3 + i] = {MNN_ALGO_WINOGRAD, kM[i], g < 2 ? MNN_OPERAND_TF32 : MNN_OPERAND_BF16, (g & 1) ? 3 : 1};
+    cands[15] = {0, 0, 0, 0};
+
+    int chunk_of[MNN_N_CANDIDATES] = {0}, nch_of[MNN_N_CANDIDATES] = {0}, pts_of[MNN_N_CANDIDATES] = {0};
+    long long ppm_of[MNN_N_CANDIDATES] = {0};
+
+    for (int i = 0; i < 15; ++i) {
+        const Cand& c = cands[i];
+        if (o.force_algo != MNN_ALGO_AUTO && o.force_algo != c.algo) continue;
+        if (c.algo == MNN_ALGO_DIRECT) {
+            if (o.operand == MNN_OPERAND_FP32_REF || o.operand == MNN_OPERAND_AUTO || o.force_algo == MNN_ALGO_DIRECT)
+                d->cost_ps[i] = direct_cost(s, cal);
+            continue;
+        }
+        if (o.operand != MNN_OPERAND_AUTO && o.operand != c.operand) continue;
+        if (o.passes != 0 && o.passes != c.passes) continue;
+        if (c.algo == MNN_ALGO_GEMM) {
+            if (s.groups != 1) continue;
+            if (o.force_m != 0) continue;
+            long long ppm = accuracy_ppm(1, s.k, 0, c.operand, c.passes);
+            if (ppm < 0) continue;
+            if ((uint64_t)ppm > gate_ppm && !(o.operand != 0 && o.force_algo == MNN_ALGO_GEMM)) continue;
+            ppm_of[i] = ppm;
+            d->cost_ps[i] = gemm_cost(s, c.operand, cal);
+            continue;
+        }
+        // Winograd
+        if (!wino_shape_ok || !winograd_supported(c.m, s.k)) continue;
+        if (o.force_m != 0 && o.force_m != c.m) continue;
+        long long ppm = 0;
+        int pid = o.points_id;
+        if (pid == MNN_POINTS_AUTO) pid = best_points(c.m, s.k, c.operand, c.passes, &ppm);
+        else ppm = accuracy_ppm(c.m, s.k, pid, c.operand, c.passes);
+        if (pid == 0 || ppm < 0) continue;
+        if ((uint64_t)ppm > gate_ppm && !fully_forced) continue;
+        pts_of[i] = pid;
+        ppm_of[i] = ppm;
+        uint64_t cost;
+        winograd_chunking(s, c.m, c.operand, c.passes, cal, &chunk_of[i], &nch_of[i], &cost);
+        d->cost_ps[i] = cost;
+    }
+
+    int best = -1;
+    for (int i = 0; i < 15; ++i)
+        if (d->cost_ps[i] != MNN_COST_INADMISSIBLE && (best < 0 || d->cost_ps[i] < d->cost_ps[best])) best = i;
+
+    // A forced combination outside the candidate list (other m, fp32 checking contraction).
+    const bool off_list = o.force_algo == MNN_ALGO_WINOGRAD && o.force_m != 0 &&
+                          (o.operand == MNN_OPERAND_FP32_REF || !(o.force_m == 2 || o.force_m == 4 || o.force_m == 6));
+    if (off_list || (best < 0 && o.force_algo == MNN_ALGO_GEMM && o.operand == MNN_OPERAND_FP32_REF)) {
+        if (o.force_algo == MNN_ALGO_WINOGRAD) {
+            if (!wino_shape_ok || !winograd_supported(o.force_m, s.k)) {
+                *err = "Winograd needs stride 1, dilation 1, groups 1, k in {2,3,5,7}, m in {2,4,6}";
+                return MNN_EUNSUPPORTED;
+            }
+            const int operand = o.operand == 0 ? MNN_OPERAND_TF32 : o.operand;
+            const int passes = o.passes == 0 ? 1 : o.passes;
+            d->algo = MNN_ALGO_WINOGRAD;
+            d->m = o.force_m;
+            d->alpha = o.force_m + s.k - 1;
+            d->operand = operand;
+            d->passes = operand == MNN_OPERAND_FP32_REF ? 1 : passes;
+            long long ppm = 0;
+            d->points_id = o.points_id ? o.points_id : best_points(d->m, s.k, operand, d->passes, &ppm);
+            d->error_ppm = accuracy_ppm(d->m, s.k, d->points_id, operand, d->passes);
+            uint64_t cost;
+            winograd_chunking(s, d->m, operand == MNN_OPERAND_FP32_REF ? MNN_OPERAND_TF32 : operand, d->passes, cal,
+                              &d->chunk_images, &d->n_chunks, &cost);
+        } else {
+            if (s.groups != 1) {
+                *err = "the GEMM scheme needs groups = 1";
+                return MNN_EUNSUPPORTED;
+            }
+            d->algo = MNN_ALGO_GEMM;
+            d->m = 1;
+            d->alpha = 1;
+            d->operand = MNN_OPERAND_FP32_REF;
+            d->passes = 1;
+            d->points_id = 0;
+            d->error_ppm = accuracy_ppm(1, s.k, 0, MNN_OPERAND_FP32_REF, 1);
+            d->chunk_images = s.N;
+            d->n_chunks = 1;
+        }
+        d->chosen = -1;
+        if (o.chunk_images > 0 && d->algo == MNN_ALGO_WINOGRAD) {
+            d->chunk_images = o.chunk_images < s.N ? o.chunk_images : s.N;
+            d->n_chunks = (s.N + d->chunk_images - 1) / d->chunk_images;
+        }
+        return MNN_OK;
+    }
+
+    if (best < 0) {
+        *err = "no scheme satisfies the forced options and the accuracy gate for this layer";
+        return MNN_EUNSUPPORTED;
+    }
+    const Cand& c = cands[best];
+    d->chosen = best;
+    d->algo = c.algo;
+    d->operand = c.operand;
+    d->passes = c.passes;
+    d->error_ppm = ppm_of[best];
+    if (c.algo == MNN_ALGO_WINOGRAD) {
+        d->m = c.m;
+        d->alpha = c.m + s.k - 1;
+        d->points_id = pts_of[best];
+        d->chunk_images = chunk_of[best];
+        d->n_chunks = nch_of[best];
+        if (o.chunk_images > 0) {
+            d->chunk_images = o.chunk_images < s.N ? o.chunk_images : s.N;
+            d->n_chunks = (s.N + d->chunk_images - 1) / d->chunk_images;
+        }
+    } else {
+        d->m = 1;
+        d->alpha = 1;
+        d->points_id = 0;
+        d->chunk_images = s.N;
+        d->n_chunks = 1;
+    }
+    return MNN_OK;
+}
+
+}  // namespace mnnb

@@ -1,0 +1,54 @@
+// Pre-inference planner: scheme selection by an integer cost model (Eq. 1-5
+// re-stated for one B200) with an accuracy gate.  Host only.
+#pragma once
+#include <cstdint>
+
+#include "../../include/mnn_conv.h"
+
+namespace mnnb {
+
+struct LayerShape {
+    int N, Cin, Cout, H, W, k, stride, pad, dil, groups, relu;
+    int OH, OW;
+};
+
+struct Calibration {
+    long long c[MNN_N_CONSTS];
+};
+
+struct Decision {
+    int algo = 0, m = 0, alpha = 0, operand = 0, passes = 0, points_id = 0;
+    int chunk_images = 0, n_chunks = 0;
+    int chosen = -1;
+    long long error_ppm = 0;
+    uint64_t cost_ps[MNN_N_CANDIDATES];
+};
+
+constexpr int kGateNumerator = 7;      // admissible when predicted error <= 0.7 x the class tolerance
+constexpr int kGateDenominator = 10;
+
+Calibration default_calibration();
+Calibration current_calibration();
+void install_calibration(const Calibration& c);
+
+// Output extent of one spatial dimension; 0 when the kernel does not fit.
+int conv_out_extent(int in, int k, int stride, int pad, int dil);
+
+// Predicted relative L2 error x 1e6 (deterministic host simulation).  m = 1 and
+// points_id = 0 gives the GEMM figure.  -1 on invalid arguments.
+long long accuracy_ppm(int m, int k, int points_id, int operand, int passes);
+
+// Best point set for (m, k, operand, passes): lowest predicted error, ties to the lower id.
+int best_points(int m, int k, int operand, int passes, long long* ppm_out);
+
+// Images per chunk and whether the chunk's V and M stay L2-resident, for a Winograd candidate.
+void winograd_chunking(const LayerShape& s, int m, int operand, int passes, const Calibration& cal,
+                       int* chunk_images, int* n_chunks, uint64_t* cost_ps);
+
+// Fills *d.  Returns MNN_OK or an mnn_status with *err set to a static reason.
+int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& cal, Decision* d, const char** err);
+
+// True when the Winograd kernels exist for (m, k).
+bool winograd_supported(int m, int k);
+
+}  // namespace mnnb
