@@ -165,6 +165,15 @@ MNN_API int mnn_conv_run_stages(mnn_conv_plan_t plan, const float* x, const floa
  * wait that ran out.  Returns MNN_OK and stores the code in *code. */
 MNN_API int mnn_conv_device_status(mnn_conv_plan_t plan, void* stream, int* code);
 
+/* Per-stage device timing.  mnn_conv_profile(plan, 1) makes every later run bracket
+ * each of its kernel launches with CUDA events on the run's stream (a small
+ * perturbation: keep it off for headline timings); 0 switches it off and frees the
+ * events.  mnn_conv_profile_read waits for the events of the LAST run and returns,
+ * per stage index (0 weight, 1 input, 2 contraction, 3 output), the summed kernel
+ * time in milliseconds and the number of launches.  Host arrays of 4. */
+MNN_API int mnn_conv_profile(mnn_conv_plan_t plan, int enable);
+MNN_API int mnn_conv_profile_read(mnn_conv_plan_t plan, float stage_ms[4], int stage_launches[4]);
+
 MNN_API void mnn_conv_destroy(mnn_conv_plan_t plan);
 
 /* Winograd generator (Eq. 8): transform matrices of F(m, k) from the chosen

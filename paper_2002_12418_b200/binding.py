@@ -25,7 +25,7 @@ OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "
 
 EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_query", "mnn_conv_set_workspace",
             "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
-            "mnn_conv_destroy", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
+            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
             "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error"]
 
 
@@ -84,6 +84,10 @@ def lib():
         L.mnn_conv_run_stages.restype = i
         L.mnn_conv_device_status.argtypes = [p, p, ctypes.POINTER(i)]
         L.mnn_conv_device_status.restype = i
+        L.mnn_conv_profile.argtypes = [p, i]
+        L.mnn_conv_profile.restype = i
+        L.mnn_conv_profile_read.argtypes = [p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i)]
+        L.mnn_conv_profile_read.restype = i
         L.mnn_conv_destroy.argtypes = [p]
         L.mnn_conv_destroy.restype = None
         L.mnn_winograd_matrices.argtypes = [i, i, i, p, p, p]
@@ -160,6 +164,18 @@ def mnn_conv_device_status(plan, stream: int) -> int:
     code = ctypes.c_int(0)
     _check(lib().mnn_conv_device_status(plan, stream, ctypes.byref(code)))
     return code.value
+
+
+def mnn_conv_profile(plan, enable: bool) -> None:
+    _check(lib().mnn_conv_profile(plan, int(bool(enable))))
+
+
+def mnn_conv_profile_read(plan):
+    """([ms per stage], [launches per stage]) of the last run; stages: weight, input, contraction, output."""
+    ms = (ctypes.c_float * 4)()
+    n = (ctypes.c_int * 4)()
+    _check(lib().mnn_conv_profile_read(plan, ms, n))
+    return list(ms), list(n)
 
 
 def mnn_conv_destroy(plan) -> None:

@@ -5,6 +5,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "../../include/mnn_conv.h"
 #include "generator.h"
@@ -51,6 +52,10 @@ struct mnn_conv_plan_s {
     long long ws_bytes = 0;
     const float* prepared_w = nullptr;
     UmmaContract uc;
+    // optional per-launch timing
+    bool profiling = false;
+    std::vector<cudaEvent_t> events;     // pairs (before, after)
+    std::vector<int> event_stage;        // stage index of each pair used by the last run
 };
 
 namespace {
@@ -110,6 +115,33 @@ void layout_workspace(mnn_conv_plan_t p)
 }
 
 bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
+
+// Brackets one launch with events when profiling is on.
+struct LaunchTimer {
+    mnn_conv_plan_t p;
+    cudaStream_t st;
+    int slot = -1;
+    LaunchTimer(mnn_conv_plan_t plan, cudaStream_t stream, int stage) : p(plan), st(stream)
+    {
+        if (!p->profiling) return;
+        const size_t used = p->event_stage.size();
+        if (2 * used + 1 >= p->events.size()) return;
+        slot = (int)used;
+        p->event_stage.push_back(stage);
+        cudaEventRecord(p->events[2 * slot], st);
+    }
+    ~LaunchTimer()
+    {
+        if (slot >= 0) cudaEventRecord(p->events[2 * slot + 1], st);
+    }
+};
+
+void free_events(mnn_conv_plan_t p)
+{
+    for (cudaEvent_t e : p->events) cudaEventDestroy(e);
+    p->events.clear();
+    p->event_stage.clear();
+}
 
 }  // namespace
 
@@ -284,6 +316,7 @@ static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, con
 static int do_weights(mnn_conv_plan_t p, const float* w, cudaStream_t st)
 {
     cudaError_t e;
+    LaunchTimer lt(p, st, 0);
     if (p->d.algo == MNN_ALGO_WINOGRAD)
         e = launch_weight_transform(w, u_hi(p), u_lo(p), p->s.Cout, p->s.Cin, p->s.k, p->d.m, p->cin_pad, p->store_mode,
                                     p->mats, st);
@@ -315,11 +348,15 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
     const LayerShape& s = p->s;
     const Decision& d = p->d;
     cudaError_t e;
+    p->event_stage.clear();
 
     if (d.algo == MNN_ALGO_DIRECT) {
         if (!(mask & MNN_STAGE_CONTRACT)) return MNN_OK;
         DirectGeom g = {s.N, s.Cin, s.Cout, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, s.groups, s.relu};
-        e = launch_direct(x, w, bias, y, g, st);
+        {
+            LaunchTimer lt(p, st, 2);
+            e = launch_direct(x, w, bias, y, g, st);
+        }
         if (e != cudaSuccess) return fail_cuda(e, "direct convolution");
         return MNN_OK;
     }
@@ -334,11 +371,13 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
         const long long T = (long long)s.N * s.OH * s.OW;
         if (mask & MNN_STAGE_INPUT) {
             GatherGeom g = {s.N, s.Cin, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, p->cin_pad};
+            LaunchTimer lt(p, st, 1);
             e = launch_gather(x, v_hi(p), v_lo(p), g, p->store_mode, st);
             if (e != cudaSuccess) return fail_cuda(e, "patch gather");
         }
         if (mask & MNN_STAGE_CONTRACT) {
             ContractEpilogue epi = {1, nullptr, 0, y, bias, s.relu, s.OH * s.OW};
+            LaunchTimer lt(p, st, 2);
             if (reference)
                 e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, 1, s.Cout, T, p->cin_pad,
                                               (long long)s.Cout * p->cin_pad, T * p->cin_pad, epi, st);
@@ -362,11 +401,13 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
         g.v_plane = p->chunk_tiles * p->cin_pad;
         g.m_row_stride = p->m_row_stride;
         if (mask & MNN_STAGE_INPUT) {
+            LaunchTimer lt(p, st, 1);
             e = launch_input_transform(x + (size_t)n0 * s.Cin * s.H * s.W, v_hi(p), v_lo(p), g, p->store_mode, p->mats, st);
             if (e != cudaSuccess) return fail_cuda(e, "input transform");
         }
         if (mask & MNN_STAGE_CONTRACT) {
             ContractEpilogue epi = {0, m_buf(p), p->m_row_stride, nullptr, nullptr, 0, 1};
+            LaunchTimer lt(p, st, 2);
             if (reference)
                 e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, alpha2, s.Cout, g.tiles,
                                               p->cin_pad, (long long)s.Cout * p->cin_pad, g.v_plane, epi, st);
@@ -375,6 +416,7 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
             if (e != cudaSuccess) return fail_cuda(e, "Winograd contraction");
         }
         if (mask & MNN_STAGE_OUTPUT) {
+            LaunchTimer lt(p, st, 3);
             e = launch_output_transform(m_buf(p), bias, y + (size_t)n0 * s.Cout * s.OH * s.OW, g, s.relu, p->mats, st);
             if (e != cudaSuccess) return fail_cuda(e, "output transform");
         }
@@ -408,7 +450,51 @@ int mnn_conv_device_status(mnn_conv_plan_t p, void* stream, int* code)
     return MNN_OK;
 }
 
-void mnn_conv_destroy(mnn_conv_plan_t p) { delete p; }
+int mnn_conv_profile(mnn_conv_plan_t p, int enable)
+{
+    if (!p) return fail(MNN_EINVAL, "NULL plan");
+    free_events(p);
+    p->profiling = false;
+    if (!enable) return MNN_OK;
+    const int pairs = p->launches_per_run + 2;
+    for (int i = 0; i < 2 * pairs; ++i) {
+        cudaEvent_t ev;
+        cudaError_t e = cudaEventCreate(&ev);
+        if (e != cudaSuccess) {
+            free_events(p);
+            return fail_cuda(e, "creating profiling events");
+        }
+        p->events.push_back(ev);
+    }
+    p->profiling = true;
+    return MNN_OK;
+}
+
+int mnn_conv_profile_read(mnn_conv_plan_t p, float stage_ms[4], int stage_launches[4])
+{
+    if (!p || !stage_ms || !stage_launches) return fail(MNN_EINVAL, "NULL argument");
+    if (!p->profiling) return fail(MNN_EINVAL, "profiling is off");
+    for (int i = 0; i < 4; ++i) {
+        stage_ms[i] = 0.0f;
+        stage_launches[i] = 0;
+    }
+    for (size_t i = 0; i < p->event_stage.size(); ++i) {
+        cudaError_t e = cudaEventSynchronize(p->events[2 * i + 1]);
+        float ms = 0.0f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, p->events[2 * i], p->events[2 * i + 1]);
+        if (e != cudaSuccess) return fail_cuda(e, "reading profiling events");
+        stage_ms[p->event_stage[i]] += ms;
+        stage_launches[p->event_stage[i]] += 1;
+    }
+    return MNN_OK;
+}
+
+void mnn_conv_destroy(mnn_conv_plan_t p)
+{
+    if (!p) return;
+    free_events(p);
+    delete p;
+}
 
 int mnn_winograd_matrices(int m, int k, int points_id, float* At, float* G, float* Bt)
 {
