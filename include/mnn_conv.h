@@ -176,6 +176,41 @@ MNN_API int mnn_conv_profile_read(mnn_conv_plan_t plan, float stage_ms[4], int s
 
 MNN_API void mnn_conv_destroy(mnn_conv_plan_t plan);
 
+/* The same forward pass as mnn_conv_run for callers that have no way to provide a
+ * workspace.  (The paper has no counterpart: its engine owns a memory pool.)
+ *
+ * Who needs it: code that is handed x, w, bias and y by somebody else and is not
+ * allowed to create device memory itself -- a plug-in running inside another
+ * framework's memory budget, a real-time loop whose rules forbid calls that may
+ * block on the driver (cudaMalloc and cudaFree synchronise the device), a process
+ * whose allocator is locked after start-up.  For them the library carries its own
+ * workspace: a fixed array of MNN_STATIC_WORKSPACE_BYTES that is part of the
+ * library image, so every GPU on which the library is loaded holds that much memory
+ * until the process exits.
+ *
+ * The plan is used for its decisions only; its own workspace (if any), prepared
+ * weights and profiling state are neither needed nor touched, and
+ * mnn_conv_set_workspace need not have been called.  The call makes no cudaMalloc,
+ * cudaFree or other allocating call.  The weights are transformed on every call
+ * (the array is shared, so nothing can be assumed to survive between calls).
+ *
+ * Limits and rules:
+ *   - plans whose info.workspace_bytes exceed MNN_STATIC_WORKSPACE_BYTES are
+ *     rejected with MNN_EWORKSPACE (nothing is launched); plan with a smaller
+ *     batch, or a smaller tile size, to fit.
+ *   - the first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - every call on a device uses the same array, which keeps the previous
+ *     call's contents; the call clears the one word that must start at zero.
+ *     Two calls that overlap on the GPU (different streams, or different
+ *     threads) race on it: serialise them.
+ *   - a bounded wait that runs out inside a kernel is recorded in the array's
+ *     status word, which this entry point does not read back.
+ * Same argument conventions, asynchrony and return codes as mnn_conv_run. */
+#define MNN_STATIC_WORKSPACE_BYTES (32u << 20)
+MNN_API int mnn_conv_run_static(mnn_conv_plan_t plan, const float* x, const float* w, const float* bias,
+                                float* y, void* stream);
+
 /* Winograd generator (Eq. 8): transform matrices of F(m, k) from the chosen
  * interpolation points plus the point at infinity, computed in exact rational
  * arithmetic and rounded once to fp32.  Host arrays, row-major:

@@ -25,7 +25,7 @@ OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "
 
 EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_query", "mnn_conv_set_workspace",
             "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
-            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
+            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
             "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error"]
 
 
@@ -80,6 +80,8 @@ def lib():
         L.mnn_conv_prepare_weights.restype = i
         L.mnn_conv_run.argtypes = [p, p, p, p, p, p]
         L.mnn_conv_run.restype = i
+        L.mnn_conv_run_static.argtypes = [p, p, p, p, p, p]
+        L.mnn_conv_run_static.restype = i
         L.mnn_conv_run_stages.argtypes = [p, p, p, p, p, p, ctypes.c_uint]
         L.mnn_conv_run_stages.restype = i
         L.mnn_conv_device_status.argtypes = [p, p, ctypes.POINTER(i)]
@@ -154,6 +156,14 @@ def mnn_conv_prepare_weights(plan, w_ptr: int, stream: int) -> None:
 
 def mnn_conv_run(plan, x_ptr: int, w_ptr: int, bias_ptr, y_ptr: int, stream: int) -> None:
     _check(lib().mnn_conv_run(plan, x_ptr, w_ptr, bias_ptr, y_ptr, stream))
+
+
+STATIC_WORKSPACE_BYTES = 32 << 20
+
+
+def mnn_conv_run_static(plan, x_ptr: int, w_ptr: int, bias_ptr, y_ptr: int, stream: int) -> None:
+    """mnn_conv_run on the library's built-in workspace (no allocation anywhere in the call)."""
+    _check(lib().mnn_conv_run_static(plan, x_ptr, w_ptr, bias_ptr, y_ptr, stream))
 
 
 def mnn_conv_run_stages(plan, x_ptr, w_ptr, bias_ptr, y_ptr, stream: int, stage_mask: int) -> None:

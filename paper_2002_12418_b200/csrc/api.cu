@@ -3,6 +3,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -534,3 +535,81 @@ int mnn_get_calibration(long long consts[MNN_N_CONSTS])
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// A run that allocates nothing: the plan's workspace is a fixed array that is
+// part of the library image on every GPU that loads it.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_workspace[MNN_STATIC_WORKSPACE_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_workspace_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the array on the current device.  In host code the array's
+// name is only a handle for the runtime, so the address is asked for once per
+// device, with that device current.
+int static_workspace_of_current_device(void** out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return fail(MNN_EUNSUPPORTED, "device index above 63");
+    std::lock_guard<std::mutex> lk(g_static_mutex);
+    if (!g_static_workspace_ptr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_workspace);
+        if (e != cudaSuccess) return fail_cuda(e, "cudaGetSymbolAddress of the built-in workspace");
+        if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 255u))
+            return fail(MNN_ECUDA, "the built-in workspace has no usable device address");
+        g_static_workspace_ptr[dev] = ptr;
+    }
+    *out = g_static_workspace_ptr[dev];
+    return MNN_OK;
+}
+
+}  // namespace
+
+extern "C" int mnn_conv_run_static(mnn_conv_plan_t p, const float* x, const float* w, const float* bias, float* y,
+                                   void* stream)
+{
+    if (!p) return fail(MNN_EINVAL, "NULL plan");
+    if (!x || !w || !y) return fail(MNN_EINVAL, "NULL tensor pointer");
+    if (p->workspace_bytes > (long long)MNN_STATIC_WORKSPACE_BYTES)
+        return fail(MNN_EWORKSPACE, "this plan needs " + std::to_string(p->workspace_bytes) +
+                                        " workspace bytes; the built-in workspace holds " +
+                                        std::to_string((long long)MNN_STATIC_WORKSPACE_BYTES));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // A private copy of the host-side plan whose workspace is the built-in array: the caller's
+    // plan (its own workspace, prepared weights, profiling state) is left untouched.
+    mnn_conv_plan_s local = *p;
+    local.profiling = false;
+    local.events.clear();
+    local.event_stage.clear();
+    local.prepared_w = nullptr;
+    local.uc.ready = false;
+    local.ws = nullptr;
+    local.ws_bytes = 0;
+    if (local.workspace_bytes > 0) {
+        void* ptr = nullptr;
+        int rc = static_workspace_of_current_device(&ptr);
+        if (rc != MNN_OK) return rc;
+        local.ws = static_cast<char*>(ptr);
+        local.ws_bytes = (long long)MNN_STATIC_WORKSPACE_BYTES;
+        // The array keeps whatever the previous call left: the status word must start at zero.
+        cudaError_t e = cudaMemsetAsync(local.ws, 0, kStatusBytes, st);
+        if (e != cudaSuccess) return fail_cuda(e, "clearing the status word");
+        if (local.d.operand != MNN_OPERAND_FP32_REF) {
+            const char* why = "";
+            const int alpha2 = local.d.algo == MNN_ALGO_WINOGRAD ? local.d.alpha * local.d.alpha : 1;
+            e = umma_contract_setup(&local.uc, local.store_mode, alpha2, local.s.Cout, local.cin_pad, local.chunk_tiles,
+                                    u_hi(&local), u_lo(&local), v_hi(&local), v_lo(&local), &why);
+            if (e != cudaSuccess)
+                return fail(MNN_ECUDA, std::string("tensor-core contraction setup: ") + why + " (" + cudaGetErrorString(e) + ")");
+        }
+    }
+    // Transformed weights are rebuilt on every call: another call may have overwritten them.
+    return mnn_conv_run_stages(&local, x, w, bias, y, stream, MNN_STAGE_ALL);
+}
