@@ -403,7 +403,8 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
         g.m_row_stride = p->m_row_stride;
         if (mask & MNN_STAGE_INPUT) {
             LaunchTimer lt(p, st, 1);
-            e = launch_input_transform(x + (size_t)n0 * s.Cin * s.H * s.W, v_hi(p), v_lo(p), g, p->store_mode, p->mats, st);
+            e = launch_input_transform(x + (size_t)n0 * s.Cin * s.H * s.W, v_hi(p), v_lo(p), g, p->store_mode, p->mats,
+                                       status_word(p), st);
             if (e != cudaSuccess) return fail_cuda(e, "input transform");
         }
         if (mask & MNN_STAGE_CONTRACT) {

@@ -180,10 +180,10 @@ extern "C" int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CO
             g.tiles = 400; g.v_plane = 400 * 64; g.m_row_stride = 416;
             float* x = reinterpret_cast<float*>(buf);
             float* V = x + (size_t)4 * 64 * 56 * 56;
-            for (int i = 0; i < 2; ++i) launch_input_transform(x, V, nullptr, g, STORE_TF32, mats, st);
+            for (int i = 0; i < 2; ++i) launch_input_transform(x, V, nullptr, g, STORE_TF32, mats, nullptr, st);
             tm.start();
             const int reps = 10;
-            for (int i = 0; i < reps; ++i) launch_input_transform(x, V, nullptr, g, STORE_TF32, mats, st);
+            for (int i = 0; i < reps; ++i) launch_input_transform(x, V, nullptr, g, STORE_TF32, mats, nullptr, st);
             ms = tm.stop();
             double t = ms / reps - launch_ms;
             if (t < ms / reps * 0.25) t = ms / reps * 0.25;

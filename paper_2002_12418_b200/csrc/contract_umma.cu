@@ -272,6 +272,39 @@ bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long 
 
 }  // namespace
 
+namespace wino {
+// Tensor map over x [images][C][H][W] (fp32) for the input transform's row copies, no swizzle; elements
+// outside the tensor read as zero.  Needs W * 4 to be a multiple of 16 bytes and a 16-byte aligned base.
+//   split_parity = false: 4-D {W, H, C, images}, box {box_w, 1, 64, 1}: 64 consecutive channels of one row.
+//   split_parity = true (C even): 5-D {W, H, 2, C/2, images}, box {box_w, 1, 1, 32, 1}: 32 channels of one
+//   parity (c = 2 * pair + parity) of one row.
+bool encode_input_map(CUtensorMap* map, const float* x, int images, int C, int H, int W, int box_w, bool split_parity)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || box_w > 256 || (W % 4) != 0 || (box_w % 4) != 0) return false;
+    const cuuint64_t plane = (cuuint64_t)H * W * 4;
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r;
+    if (split_parity) {
+        if (C % 2) return false;
+        const cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, 2, (cuuint64_t)(C / 2), (cuuint64_t)images};
+        const cuuint64_t strides[4] = {(cuuint64_t)W * 4, plane, 2 * plane, (cuuint64_t)C * plane};
+        const cuuint32_t box[5] = {(cuuint32_t)box_w, 1, 1, 32, 1};
+        r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[4] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)C, (cuuint64_t)images};
+        const cuuint64_t strides[3] = {(cuuint64_t)W * 4, plane, (cuuint64_t)C * plane};
+        const cuuint32_t box[4] = {(cuuint32_t)box_w, 1, 64, 1};
+        r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    return r == CUDA_SUCCESS;
+}
+}  // namespace wino
+
 cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout, int cin_pad, long long tiles_capacity,
                                 void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why)
 {

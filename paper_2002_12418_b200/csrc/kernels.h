@@ -41,9 +41,10 @@ cudaError_t launch_weight_transform(const float* w, void* U_hi, void* U_lo, int 
 // GEMM scheme: rounded copy of w [Cout][Cin*k*k] into U [Cout][k_pad].
 cudaError_t launch_weight_round(const float* w, void* U_hi, void* U_lo, int Cout, int Kd, int k_pad, int mode,
                                 cudaStream_t stream);
-// V = B^T d B for every tile of the chunk.  x points at the chunk's first image.
+// V = B^T d B for every tile of the chunk.  x points at the chunk's first image.  `status` (device, may be
+// NULL) receives a code if a bounded wait inside the kernel runs out.
 cudaError_t launch_input_transform(const float* x, void* V_hi, void* V_lo, const WinoGeom& g, int mode,
-                                   const TransformMatrices& mats, cudaStream_t stream);
+                                   const TransformMatrices& mats, int* status, cudaStream_t stream);
 // y = act(A^T M A + bias).  y points at the chunk's first image.
 cudaError_t launch_output_transform(const float* M, const float* bias, float* y, const WinoGeom& g, int relu,
                                     const TransformMatrices& mats, cudaStream_t stream);

@@ -1,0 +1,461 @@
+// Winograd input transform V = B^T d B (Eq. 6) as a persistent, warp-specialised kernel.
+//
+// Work item = (image, tile row, segment of up to `txs` tiles of that row, block of 64
+// channels).  The alpha input rows of an item are staged in a ring of shared-memory
+// buffers laid out [row][channel slot][column]; the number of staged columns `wb` is an
+// odd multiple of 4 words, so that 32 lanes reading 128-bit vectors from 32 consecutive
+// slots touch every bank once.  When the image rows are 16-byte aligned (W a multiple of
+// 4) one loader warp issues TMA box copies, one per input row (box = 64 channels x wb
+// columns; or two boxes of 32 channels, even and odd, through a 5-D view of x that splits
+// the channel parity); everything outside the image, including the zero padding of the
+// convolution and channels beyond Cin, arrives as zeros, so several items are in flight
+// with no load instructions at all.  Otherwise four loader warps issue contiguous cp.async
+// copies with explicit zero fill.  The remaining warps take (item, tile) units in order.  A
+// lane transforms one tile of TWO adjacent channels held as packed fp32 pairs (packed
+// fp32x2 multiply-adds), or of one channel for alpha >= 8 where a pair would not fit the
+// register file, and writes one 128- or 256-byte row piece of V[xi][tile][channel] per
+// warp store.
+//
+// When the interpolation points are symmetric (0, +-p1, +-p2, ..., infinity; alpha even)
+// B^T has a fixed zero pattern and its +p / -p rows share coefficients up to sign
+// (the generator polynomial of Eq. 8 is odd), so each 1-D pass needs about half the
+// multiplies of the dense form.  The host checks the pattern on the generated matrix
+// and otherwise selects the dense form.
+//
+// Loader and compute warps hand buffers over through mbarriers; every wait is bounded
+// and reports through the plan's status word instead of hanging.
+#pragma once
+#include <cuda_bf16.h>
+
+#include <cstring>
+#include <type_traits>
+
+#include "kernels.h"
+#include "umma.cuh"
+
+namespace mnnb {
+namespace wino {
+
+constexpr int kItChannels = 64;         // channels per work item
+constexpr int kItWarps = 16;
+constexpr int kItThreads = 32 * kItWarps;
+constexpr int kItMaxBuffers = 6;
+constexpr int kItSmemBudget = 200 * 1024;
+constexpr int kErrInputLoaderWait = 11, kErrInputComputeWait = 12;
+
+struct MatBt2 { float2 v[12 * 12]; };   // B^T with every entry duplicated into a pair
+
+struct InputItems {
+    int txs;            // tiles per item
+    int nseg;           // segments per tile row
+    int wb;             // staged columns per channel row: 4 x odd words
+    int nbuf;           // ring depth
+    int cblocks;        // blocks of 64 channels
+    int use_tma;        // 1: TMA box copies (W % 4 == 0), 0: cp.async
+    int vec;            // alignment of the staged column grid in elements: 4 with TMA, else 2 or 1
+    int loader_warps;   // 1 with TMA, else 4
+    int buf_words;      // words per buffer = alpha * 64 * wb
+    long long n_items;
+};
+
+__device__ __forceinline__ float round_tf32_v(float v)
+{
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(v));
+    return __uint_as_float(u);
+}
+
+// ---- value types: one channel (float) or two adjacent channels (float2) per lane ----
+__device__ __forceinline__ float v_mul(float2 c, float a) { return c.x * a; }
+__device__ __forceinline__ float v_fma(float2 c, float a, float acc) { return fmaf(c.x, a, acc); }
+__device__ __forceinline__ float v_add(float a, float b) { return a + b; }
+__device__ __forceinline__ float v_sub(float a, float b) { return a - b; }
+__device__ __forceinline__ float2 v_mul(float2 c, float2 a) { return __fmul2_rn(c, a); }
+__device__ __forceinline__ float2 v_fma(float2 c, float2 a, float2 acc) { return __ffma2_rn(c, a, acc); }
+__device__ __forceinline__ float2 v_add(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 v_sub(float2 a, float2 b) { return __ffma2_rn(make_float2(-1.0f, -1.0f), b, a); }
+__device__ __forceinline__ float v_make(float a, float, float) { return a; }
+__device__ __forceinline__ float2 v_make(float a, float b, float2) { return make_float2(a, b); }
+
+// One 1-D pass o = B^T d.  SYM: the symmetric-point structure described above.
+template <int ALPHA, bool SYM, typename T>
+__device__ __forceinline__ void pass_1d(const T (&d)[ALPHA], T (&o)[ALPHA], const MatBt2& Bt)
+{
+    if (SYM) {
+        // row of the point 0: even powers only
+        T s = v_mul(Bt.v[0], d[0]);
+#pragma unroll
+        for (int r = 2; r < ALPHA; r += 2) s = v_fma(Bt.v[r], d[r], s);
+        o[0] = s;
+        // row of the point at infinity: odd powers only
+        s = v_mul(Bt.v[(ALPHA - 1) * ALPHA + 1], d[1]);
+#pragma unroll
+        for (int r = 3; r < ALPHA; r += 2) s = v_fma(Bt.v[(ALPHA - 1) * ALPHA + r], d[r], s);
+        o[ALPHA - 1] = s;
+        // +p / -p pairs: even part E (r = 2, 4, ..), odd part O (r = 1, 3, ..); rows are E + O and E - O
+#pragma unroll
+        for (int p = 1; p < ALPHA - 1; p += 2) {
+            T e = v_mul(Bt.v[p * ALPHA + 2], d[2]);
+#pragma unroll
+            for (int r = 4; r < ALPHA - 1; r += 2) e = v_fma(Bt.v[p * ALPHA + r], d[r], e);
+            T od = v_mul(Bt.v[p * ALPHA + 1], d[1]);
+#pragma unroll
+            for (int r = 3; r < ALPHA - 1; r += 2) od = v_fma(Bt.v[p * ALPHA + r], d[r], od);
+            o[p] = v_add(e, od);
+            o[p + 1] = v_sub(e, od);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < ALPHA; ++i) {
+            T s = v_mul(Bt.v[i * ALPHA], d[0]);
+#pragma unroll
+            for (int r = 1; r < ALPHA; ++r) s = v_fma(Bt.v[i * ALPHA + r], d[r], s);
+            o[i] = s;
+        }
+    }
+}
+
+// ---- stores in the operand formats (lane's channel, or channel pair, at byte pointers hi / lo) ----
+template <int MODE>
+__device__ __forceinline__ void put(char* hi, char* lo, float v)
+{
+    if (MODE == STORE_TF32) {
+        *reinterpret_cast<float*>(hi) = round_tf32_v(v);
+    } else if (MODE == STORE_BF16) {
+        *reinterpret_cast<__nv_bfloat16*>(hi) = __float2bfloat16_rn(v);
+    } else if (MODE == STORE_TF32_SPLIT) {
+        const float h = round_tf32_v(v);
+        *reinterpret_cast<float*>(hi) = h;
+        *reinterpret_cast<float*>(lo) = round_tf32_v(v - h);
+    } else if (MODE == STORE_BF16_SPLIT) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        *reinterpret_cast<__nv_bfloat16*>(hi) = h;
+        *reinterpret_cast<__nv_bfloat16*>(lo) = __float2bfloat16_rn(v - __bfloat162float(h));
+    } else {
+        *reinterpret_cast<float*>(hi) = v;
+    }
+}
+template <int MODE>
+__device__ __forceinline__ void put(char* hi, char* lo, float2 v)
+{
+    if (MODE == STORE_TF32) {
+        *reinterpret_cast<float2*>(hi) = make_float2(round_tf32_v(v.x), round_tf32_v(v.y));
+    } else if (MODE == STORE_BF16) {
+        *reinterpret_cast<__nv_bfloat162*>(hi) = __floats2bfloat162_rn(v.x, v.y);
+    } else if (MODE == STORE_TF32_SPLIT) {
+        const float2 h = make_float2(round_tf32_v(v.x), round_tf32_v(v.y));
+        *reinterpret_cast<float2*>(hi) = h;
+        const float2 l = v_sub(v, h);
+        *reinterpret_cast<float2*>(lo) = make_float2(round_tf32_v(l.x), round_tf32_v(l.y));
+    } else if (MODE == STORE_BF16_SPLIT) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(v.x, v.y);
+        const float2 l = v_sub(v, __bfloat1622float2(h));
+        *reinterpret_cast<__nv_bfloat162*>(hi) = h;
+        *reinterpret_cast<__nv_bfloat162*>(lo) = __floats2bfloat162_rn(l.x, l.y);
+    } else {
+        *reinterpret_cast<float2*>(hi) = v;
+    }
+}
+
+// Row pass of one tile: h[r][j'] = sum_j d[r][j] Bt[j'][j].  p0 (and p1 for the second channel of a pair)
+// point at the 16-byte aligned vector of staged row 0 that holds the tile's first column; OFF = that
+// column's index in the vector; row_words = words between staged rows.
+template <int ALPHA, bool SYM, int OFF, typename T>
+__device__ __forceinline__ void rows_pass(const float* p0, const float* p1, int row_words, const MatBt2& Bt,
+                                          T (&h)[ALPHA][ALPHA])
+{
+    constexpr int NV = (OFF + ALPHA + 3) / 4;
+    constexpr bool kPair = std::is_same<T, float2>::value;
+#pragma unroll
+    for (int r = 0; r < ALPHA; ++r) {
+        float a[4 * NV], b[4 * NV];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const float4 q = *reinterpret_cast<const float4*>(p0 + r * row_words + 4 * v);
+            a[4 * v] = q.x; a[4 * v + 1] = q.y; a[4 * v + 2] = q.z; a[4 * v + 3] = q.w;
+            if (kPair) {
+                const float4 s = *reinterpret_cast<const float4*>(p1 + r * row_words + 4 * v);
+                b[4 * v] = s.x; b[4 * v + 1] = s.y; b[4 * v + 2] = s.z; b[4 * v + 3] = s.w;
+            } else {
+                b[4 * v] = b[4 * v + 1] = b[4 * v + 2] = b[4 * v + 3] = 0.0f;
+            }
+        }
+        T d[ALPHA];
+#pragma unroll
+        for (int j = 0; j < ALPHA; ++j) d[j] = v_make(a[OFF + j], b[OFF + j], T());
+        pass_1d<ALPHA, SYM, T>(d, h[r], Bt);
+    }
+}
+
+// Column pass and stores: V[i][j] = sum_r Bt[i][r] h[r][j], transform position xi = i * alpha + j.
+template <int ALPHA, bool SYM, int MODE, typename T>
+__device__ __forceinline__ void cols_pass_store(const T (&h)[ALPHA][ALPHA], const MatBt2& Bt, char* hi, char* lo,
+                                                long long plane_bytes)
+{
+    const long long row_step = plane_bytes * ALPHA;   // from transform position (i, j) to (i + 1, j)
+#pragma unroll
+    for (int j = 0; j < ALPHA; ++j) {
+        T col[ALPHA], o[ALPHA];
+#pragma unroll
+        for (int r = 0; r < ALPHA; ++r) col[r] = h[r][j];
+        pass_1d<ALPHA, SYM, T>(col, o, Bt);
+        char* ph = hi;
+        char* pl = lo;
+#pragma unroll
+        for (int i = 0; i < ALPHA; ++i) {
+            put<MODE>(ph, pl, o[i]);
+            ph += row_step;
+            pl += row_step;
+        }
+        hi += plane_bytes;
+        lo += plane_bytes;
+    }
+}
+
+// Shared-memory slot of channel c (0..63) of an item.  With channel pairs, lane l works on channels
+// 2l and 2l + 1 and finds them in slots l and 32 + l, so that both reads walk consecutive slots.
+template <bool PAIR>
+__device__ __forceinline__ int slot_of(int c)
+{
+    return PAIR ? ((c & 1) * 32 + (c >> 1)) : c;
+}
+
+template <int ALPHA, bool SYM, bool PAIR>
+__global__ void __launch_bounds__(kItThreads, 1)
+input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ CUtensorMap xmap, char* V_hi, char* V_lo,
+                          WinoGeom g, InputItems it, int mode, const __grid_constant__ MatBt2 Bt, int* status)
+{
+    extern __shared__ __align__(128) float s_buf[];
+    __shared__ __align__(8) uint64_t full_bar[kItMaxBuffers];
+    __shared__ __align__(8) uint64_t empty_bar[kItMaxBuffers];
+    __shared__ int4 item_desc[kItMaxBuffers];      // (image, tile row, first tile, channel block) of the item in each buffer
+    __shared__ int abort_flag;
+    volatile int* abortp = &abort_flag;
+    using T = typename std::conditional<PAIR, float2, float>::type;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kHalves = PAIR ? 1 : 2;                 // units per tile: one for 64 channels, or two of 32
+    const int units_per_item = it.txs * kHalves;
+    const int n_compute = kItWarps - it.loader_warps;
+    const int row_words = kItChannels * it.wb;            // words between staged rows
+    if (threadIdx.x == 0) {
+        for (int b = 0; b < it.nbuf; ++b) {
+            ptx::mbar_init(ptx::smem_u32(&full_bar[b]), it.use_tma ? 1u : 32u * (uint32_t)it.loader_warps);
+            ptx::mbar_init(ptx::smem_u32(&empty_bar[b]), (uint32_t)units_per_item);
+        }
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+        if (it.use_tma) ptx::prefetch_tensormap(&xmap);
+    }
+    __syncthreads();
+
+    // items of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ... (32-bit: the host keeps n_items below 2^31)
+    const unsigned first = blockIdx.x, n_items = (unsigned)it.n_items;
+    const unsigned n_local = first < n_items ? (n_items - first + gridDim.x - 1) / gridDim.x : 0;
+    const int eb = (mode == STORE_BF16 || mode == STORE_BF16_SPLIT) ? 2 : 4;
+
+    if (warp < it.loader_warps) {
+        // ------------------------------- loaders -------------------------------
+        int b = 0;
+        uint32_t round = 0;
+        for (unsigned li = 0; li < n_local; ++li) {
+            if (round > 0 && !ptx::mbar_wait_relaxed(ptx::smem_u32(&empty_bar[b]), (round - 1) & 1u, abortp)) {
+                if (!*abortp && status) atomicCAS(status, 0, kErrInputLoaderWait);
+                *abortp = 1;
+                break;
+            }
+            unsigned item = first + li * gridDim.x;
+            const int cb = (int)(item % (unsigned)it.cblocks); item /= (unsigned)it.cblocks;
+            const int seg = (int)(item % (unsigned)it.nseg); item /= (unsigned)it.nseg;
+            const int ty = (int)(item % (unsigned)g.th);
+            const int img = (int)(item / (unsigned)g.th);
+            const int tx0 = seg * it.txs;
+            const int ih0 = ty * g.m - g.pad, iw0 = tx0 * g.m - g.pad;
+            const int a0 = iw0 - ((iw0 % it.vec + it.vec) % it.vec);      // first staged column, on the vector grid
+            const int c0 = cb * kItChannels;
+            if (threadIdx.x == 0) item_desc[b] = make_int4(img, ty, tx0, cb);
+            const uint32_t sbuf = ptx::smem_u32(s_buf) + (uint32_t)b * (uint32_t)it.buf_words * 4u;
+            const uint32_t bar = ptx::smem_u32(&full_bar[b]);
+            if (it.use_tma) {
+                if (lane == 0) ptx::mbar_expect_tx(bar, (uint32_t)it.buf_words * 4u);
+                __syncwarp();
+                if (PAIR) {
+                    // lane = (row, parity): 32 channels of one parity of one input row
+                    if (lane < 2 * ALPHA) {
+                        const int r = lane >> 1, par = lane & 1;
+                        ptx::tma_load_5d(sbuf + (uint32_t)(r * row_words + par * 32 * it.wb) * 4u, &xmap, bar, a0, ih0 + r, par,
+                                         c0 >> 1, img);
+                    }
+                } else {
+                    if (lane < ALPHA) ptx::tma_load_4d(sbuf + (uint32_t)(lane * row_words) * 4u, &xmap, bar, a0, ih0 + lane, c0, img);
+                }
+            } else {
+                // contiguous copies: consecutive lanes take consecutive staged elements of one (channel, row)
+                const float* ximg = x + (size_t)img * g.Cin * g.H * g.W;
+                const int per_row = it.wb / it.vec;                        // copies per staged row
+                const int per_ch = ALPHA * per_row;
+                const int total = kItChannels * per_ch;
+                for (int e = warp * 32 + lane; e < total; e += 32 * it.loader_warps) {
+                    const int c = e / per_ch, rem = e - c * per_ch;
+                    const int r = rem / per_row, jv = rem - r * per_row;
+                    const int ih = ih0 + r, iw = a0 + jv * it.vec, ci = c0 + c;
+                    const uint32_t dst = sbuf + (uint32_t)(r * row_words + slot_of<PAIR>(c) * it.wb + jv * it.vec) * 4u;
+                    const bool ok = ih >= 0 && ih < g.H && ci < g.Cin && iw >= 0 && iw + it.vec <= g.W;
+                    const float* src = ok ? ximg + ((size_t)ci * g.H + ih) * g.W + iw : ximg;
+                    if (it.vec == 2) ptx::cp_async_8(dst, src, ok ? 8u : 0u);
+                    else ptx::cp_async_4(dst, src, ok ? 4u : 0u);
+                }
+                ptx::cp_async_arrive_noinc(bar);
+            }
+            if (++b == it.nbuf) {
+                b = 0;
+                ++round;
+            }
+        }
+        if (!it.use_tma) ptx::cp_async_wait_all();
+    } else {
+        // ------------------------------- compute -------------------------------
+        const int cw = warp - it.loader_warps;
+        const long long plane_bytes = (long long)g.v_plane * eb;
+        // this warp's units: cw, cw + n_compute, ... of the CTA's (item, tile[, half]) sequence, tracked incrementally
+        unsigned li = 0;
+        int within = cw, b = 0;
+        uint32_t round = 0;
+        for (;;) {
+            while (within >= units_per_item) {
+                within -= units_per_item;
+                ++li;
+                if (++b == it.nbuf) {
+                    b = 0;
+                    ++round;
+                }
+            }
+            if (li >= n_local) break;
+            const int t = PAIR ? within : (within >> 1), half = PAIR ? 0 : (within & 1);
+            if (!ptx::mbar_wait_relaxed(ptx::smem_u32(&full_bar[b]), round & 1u, abortp)) {
+                if (!*abortp && status) atomicCAS(status, 0, kErrInputComputeWait);
+                *abortp = 1;
+                break;
+            }
+            const int4 desc = item_desc[b];
+            const int img = desc.x, ty = desc.y, tx0 = desc.z, cb = desc.w;
+            const int tx = tx0 + t;
+            const int c = cb * kItChannels + (PAIR ? 2 * lane : half * 32 + lane);
+            if (tx < g.tw && c < g.cin_pad) {
+                const long long tile = ((long long)img * g.th + ty) * g.tw + tx;
+                const int iw0 = tx0 * g.m - g.pad;
+                const int s0 = (iw0 % it.vec + it.vec) % it.vec + t * g.m;     // staged column of the tile's first input column
+                const float* p0 = s_buf + (size_t)b * it.buf_words + (size_t)(PAIR ? lane : half * 32 + lane) * it.wb + (s0 & ~3);
+                const float* p1 = p0 + 32 * it.wb;
+                T h[ALPHA][ALPHA];
+                switch (s0 & 3) {
+                    case 0: rows_pass<ALPHA, SYM, 0, T>(p0, p1, row_words, Bt, h); break;
+                    case 1: rows_pass<ALPHA, SYM, 1, T>(p0, p1, row_words, Bt, h); break;
+                    case 2: rows_pass<ALPHA, SYM, 2, T>(p0, p1, row_words, Bt, h); break;
+                    default: rows_pass<ALPHA, SYM, 3, T>(p0, p1, row_words, Bt, h); break;
+                }
+                const long long off = (tile * g.cin_pad + c) * eb;
+                char* hi = V_hi + off;
+                char* lo = V_lo ? V_lo + off : nullptr;
+                switch (mode) {
+                    case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T>(h, Bt, hi, lo, plane_bytes); break;
+                    case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T>(h, Bt, hi, lo, plane_bytes); break;
+                    case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
+                    case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
+                    default: cols_pass_store<ALPHA, SYM, STORE_FP32, T>(h, Bt, hi, lo, plane_bytes); break;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[b]));
+            within += n_compute;
+        }
+    }
+}
+
+// True when Bt (alpha x alpha, row-major) has the zero pattern and the +p / -p row symmetry
+// that pass_1d<.., SYM = true> assumes.
+inline bool bt_has_symmetric_structure(const float* Bt, int alpha)
+{
+    if (alpha < 4 || (alpha & 1)) return false;
+    for (int r = 0; r < alpha; ++r) {
+        if ((r & 1) && Bt[r] != 0.0f) return false;                                  // point 0: even powers only
+        if (!(r & 1) && Bt[(alpha - 1) * alpha + r] != 0.0f) return false;            // infinity: odd powers only
+    }
+    for (int p = 1; p < alpha - 1; p += 2) {
+        const float* a = Bt + p * alpha;
+        const float* b = Bt + (p + 1) * alpha;
+        if (a[0] != 0.0f || b[0] != 0.0f || a[alpha - 1] != 0.0f || b[alpha - 1] != 0.0f) return false;
+        for (int r = 1; r < alpha - 1; ++r)
+            if (b[r] != ((r & 1) ? -a[r] : a[r])) return false;
+    }
+    return true;
+}
+
+// Item geometry: the longest segment for which at least three buffers fit shared memory.
+inline bool plan_input_items(const WinoGeom& g, int alpha, bool tma_ok, InputItems* it)
+{
+    it->use_tma = tma_ok ? 1 : 0;
+    it->vec = tma_ok ? 4 : ((g.W % 2 == 0) ? 2 : 1);
+    it->loader_warps = tma_ok ? 1 : 4;
+    it->cblocks = (g.cin_pad + kItChannels - 1) / kItChannels;
+    for (int nseg = 1; nseg <= g.tw; ++nseg) {
+        const int txs = (g.tw + nseg - 1) / nseg;
+        const int span = (txs - 1) * g.m + alpha;
+        // staged columns: the span, what the vector grid adds in front (up to vec - 1) and what the compute
+        // side may read beyond the last tile (whole 4-wide vectors), rounded up to 4 x odd
+        int wb = (span + (it->vec - 1) + 3 + 3) / 4 * 4;
+        if (((wb / 4) & 1) == 0) wb += 4;
+        if (wb > 256) continue;
+        const long long bytes = (long long)alpha * kItChannels * wb * 4;
+        long long nbuf = kItSmemBudget / bytes;
+        if (nbuf >= 3 || txs == 1) {
+            if (nbuf < 2) return false;
+            if (nbuf > kItMaxBuffers) nbuf = kItMaxBuffers;
+            it->txs = txs;
+            it->nseg = (g.tw + txs - 1) / txs;
+            it->wb = wb;
+            it->nbuf = (int)nbuf;
+            it->buf_words = alpha * kItChannels * wb;
+            it->n_items = (long long)g.images * g.th * it->nseg * it->cblocks;
+            return it->n_items < (1ll << 31);
+        }
+    }
+    return false;
+}
+
+// Defined beside the other tensor-map code (contract_umma.cu).
+bool encode_input_map(CUtensorMap* map, const float* x, int images, int C, int H, int W, int box_w, bool split_parity);
+
+template <int ALPHA>
+cudaError_t launch_input_ws(const float* x, void* V_hi, void* V_lo, const WinoGeom& g, int mode, const TransformMatrices& mats,
+                            int* status, int num_sms, cudaStream_t stream)
+{
+    MatBt2 bt;
+    for (int i = 0; i < ALPHA * ALPHA; ++i) bt.v[i] = make_float2(mats.Bt[i], mats.Bt[i]);
+    const bool sym = bt_has_symmetric_structure(mats.Bt, ALPHA);
+    constexpr bool kPair = ALPHA <= 6;
+    InputItems it;
+    bool tma_ok = (g.W % 4 == 0) && ((reinterpret_cast<uintptr_t>(x) & 15u) == 0) && (!kPair || g.Cin % 2 == 0);
+    CUtensorMap xmap;
+    std::memset(&xmap, 0, sizeof(xmap));
+    if (tma_ok) {
+        if (!plan_input_items(g, ALPHA, true, &it) || !encode_input_map(&xmap, x, g.images, g.Cin, g.H, g.W, it.wb, kPair))
+            tma_ok = false;
+    }
+    if (!tma_ok && !plan_input_items(g, ALPHA, false, &it)) return cudaErrorInvalidConfiguration;
+    const size_t smem = (size_t)it.nbuf * it.buf_words * sizeof(float);
+    long long grid = it.n_items < num_sms ? it.n_items : num_sms;
+    if (grid <= 0) return cudaSuccess;
+    auto launch = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kItSmemBudget);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)grid, kItThreads, smem, stream>>>(x, xmap, static_cast<char*>(V_hi), static_cast<char*>(V_lo), g, it,
+                                                           mode, bt, status);
+        return cudaGetLastError();
+    };
+    if (sym) return launch(input_transform_ws_kernel<ALPHA, true, kPair>);
+    return launch(input_transform_ws_kernel<ALPHA, false, kPair>);
+}
+
+}  // namespace wino
+}  // namespace mnnb

@@ -128,17 +128,25 @@ cudaError_t launch_weight_round(const float* w, void* U_hi, void* U_lo, int Cout
 }
 
 cudaError_t launch_input_transform(const float* x, void* V_hi, void* V_lo, const WinoGeom& g, int mode,
-                                   const TransformMatrices& mats, cudaStream_t stream)
+                                   const TransformMatrices& mats, int* status, cudaStream_t stream)
 {
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            n <= 0)
+            n = 148;
+        num_sms = n;
+    }
     switch (g.alpha) {
-        case 3: return MNNB_INPUT_FN(3)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 4: return MNNB_INPUT_FN(4)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 5: return MNNB_INPUT_FN(5)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 6: return MNNB_INPUT_FN(6)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 7: return MNNB_INPUT_FN(7)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 8: return MNNB_INPUT_FN(8)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 10: return MNNB_INPUT_FN(10)(x, V_hi, V_lo, g, mode, mats, stream);
-        case 12: return MNNB_INPUT_FN(12)(x, V_hi, V_lo, g, mode, mats, stream);
+        case 3: return MNNB_INPUT_FN(3)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 4: return MNNB_INPUT_FN(4)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 5: return MNNB_INPUT_FN(5)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 6: return MNNB_INPUT_FN(6)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 7: return MNNB_INPUT_FN(7)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 8: return MNNB_INPUT_FN(8)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 10: return MNNB_INPUT_FN(10)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
+        case 12: return MNNB_INPUT_FN(12)(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream);
         default: return cudaErrorInvalidValue;
     }
 }

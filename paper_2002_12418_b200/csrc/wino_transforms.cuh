@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "wino_input.cuh"
 
 namespace mnnb {
 namespace wino {
@@ -44,80 +45,6 @@ __device__ __forceinline__ void store_operand(void* hi, void* lo, size_t idx, fl
         default:
             reinterpret_cast<float*>(hi)[idx] = v;
             break;
-    }
-}
-
-// ---------------------------------------------------------------------------
-// Input transform.  One CTA = one tile row of one image x 32 channels.  The
-// alpha input rows are staged in shared memory ([channel][row][column], channel
-// stride odd so that a warp reading 32 channels at one position hits 32 banks);
-// then each thread transforms one (tile, channel) in registers and writes the
-// alpha^2 results with the channel index fastest, i.e. 128 contiguous bytes per
-// warp store into V[xi][tile][channel].
-// ---------------------------------------------------------------------------
-constexpr int kInChannels = 32;
-constexpr int kInThreads = 256;
-
-template <int ALPHA>
-__global__ void __launch_bounds__(kInThreads) input_transform_kernel(const float* __restrict__ x, void* V_hi, void* V_lo,
-                                                                      WinoGeom g, int mode, MatBt Bt)
-{
-    extern __shared__ float s_in[];
-    const int ws = (g.tw - 1) * g.m + ALPHA;                 // staged row width
-    const int cs = (ALPHA * ws) | 1;                         // channel stride (odd)
-    const int img = blockIdx.x / g.th, ty = blockIdx.x % g.th;
-    const int c0 = blockIdx.y * kInChannels;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    // stage: one warp per (channel, row)
-    for (int row = warp; row < kInChannels * ALPHA; row += kInThreads / 32) {
-        const int c = row / ALPHA, r = row % ALPHA;
-        const int ci = c0 + c;
-        const int ih = ty * g.m - g.pad + r;
-        const bool row_ok = ci < g.Cin && ih >= 0 && ih < g.H;
-        const float* src = x + (((size_t)img * g.Cin + (row_ok ? ci : 0)) * g.H + (row_ok ? ih : 0)) * g.W;
-        float* dst = s_in + c * cs + r * ws;
-        for (int j = lane; j < ws; j += 32) {
-            const int iw = j - g.pad;
-            dst[j] = (row_ok && iw >= 0 && iw < g.W) ? __ldg(src + iw) : 0.0f;
-        }
-    }
-    __syncthreads();
-
-    const int items = kInChannels * g.tw;
-    for (int item = threadIdx.x; item < items; item += kInThreads) {
-        const int c = item & (kInChannels - 1), tx = item / kInChannels;
-        const int ci = c0 + c;
-        if (ci >= g.cin_pad) continue;
-        float d[ALPHA][ALPHA];
-        const float* src = s_in + c * cs + tx * g.m;
-#pragma unroll
-        for (int r = 0; r < ALPHA; ++r)
-#pragma unroll
-            for (int j = 0; j < ALPHA; ++j) d[r][j] = src[r * ws + j];
-        // t = B^T d
-        float t[ALPHA][ALPHA];
-#pragma unroll
-        for (int i = 0; i < ALPHA; ++i)
-#pragma unroll
-            for (int j = 0; j < ALPHA; ++j) {
-                float s = 0.0f;
-#pragma unroll
-                for (int r = 0; r < ALPHA; ++r) s = fmaf(Bt.v[i * ALPHA + r], d[r][j], s);
-                t[i][j] = s;
-            }
-        const long long tile = ((long long)img * g.th + ty) * g.tw + tx;
-        const size_t base = (size_t)tile * g.cin_pad + ci;
-        // V = t B, written as it is produced
-#pragma unroll
-        for (int i = 0; i < ALPHA; ++i)
-#pragma unroll
-            for (int j = 0; j < ALPHA; ++j) {
-                float s = 0.0f;
-#pragma unroll
-                for (int r = 0; r < ALPHA; ++r) s = fmaf(t[i][r], Bt.v[j * ALPHA + r], s);
-                store_operand(V_hi, V_lo, (size_t)(i * ALPHA + j) * g.v_plane + base, s, mode);
-            }
     }
 }
 
@@ -185,26 +112,6 @@ __global__ void __launch_bounds__(kOutThreads) output_transform_kernel(const flo
     }
 }
 
-template <int ALPHA>
-cudaError_t launch_input_alpha(const float* x, void* V_hi, void* V_lo, const WinoGeom& g, int mode,
-                               const TransformMatrices& mats, cudaStream_t stream)
-{
-    MatBt bt;
-    for (int i = 0; i < ALPHA * ALPHA; ++i) bt.v[i] = mats.Bt[i];
-    const int ws = (g.tw - 1) * g.m + ALPHA;
-    const int cs = (ALPHA * ws) | 1;
-    const size_t smem = (size_t)kInChannels * cs * sizeof(float);
-    if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
-    auto kern = input_transform_kernel<ALPHA>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    dim3 grid((unsigned)(g.images * g.th), (unsigned)((g.cin_pad + kInChannels - 1) / kInChannels));
-    kern<<<grid, kInThreads, smem, stream>>>(x, V_hi, V_lo, g, mode, bt);
-    return cudaGetLastError();
-}
-
 template <int ALPHA, int M>
 cudaError_t launch_output_am(const float* Mx, const float* bias, float* y, const WinoGeom& g, int relu,
                              const TransformMatrices& mats, cudaStream_t stream)
@@ -223,10 +130,10 @@ cudaError_t launch_output_am(const float* Mx, const float* bias, float* y, const
 // One non-template entry point per instantiation, defined in wino_inst_*.cu.
 #define MNNB_INPUT_FN(A) launch_input_transform_a##A
 #define MNNB_OUTPUT_FN(A, MM) launch_output_transform_a##A##_m##MM
-#define MNNB_INPUT_ARGS const float *x, void *V_hi, void *V_lo, const WinoGeom &g, int mode, const TransformMatrices &mats, cudaStream_t stream
+#define MNNB_INPUT_ARGS const float *x, void *V_hi, void *V_lo, const WinoGeom &g, int mode, const TransformMatrices &mats, int *status, int num_sms, cudaStream_t stream
 #define MNNB_OUTPUT_ARGS const float *Mx, const float *bias, float *y, const WinoGeom &g, int relu, const TransformMatrices &mats, cudaStream_t stream
 #define MNNB_DEFINE_INPUT(A) \
-    namespace mnnb { cudaError_t MNNB_INPUT_FN(A)(MNNB_INPUT_ARGS) { return wino::launch_input_alpha<A>(x, V_hi, V_lo, g, mode, mats, stream); } }
+    namespace mnnb { cudaError_t MNNB_INPUT_FN(A)(MNNB_INPUT_ARGS) { return wino::launch_input_ws<A>(x, V_hi, V_lo, g, mode, mats, status, num_sms, stream); } }
 #define MNNB_DEFINE_OUTPUT(A, MM) \
     namespace mnnb { cudaError_t MNNB_OUTPUT_FN(A, MM)(MNNB_OUTPUT_ARGS) { return wino::launch_output_am<A, MM>(Mx, bias, y, g, relu, mats, stream); } }
 #define MNNB_DECLARE_INPUT(A) namespace mnnb { cudaError_t MNNB_INPUT_FN(A)(MNNB_INPUT_ARGS); }
