@@ -241,7 +241,7 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
     if (threadIdx.x == 0) {
         for (int b = 0; b < it.nbuf; ++b) {
             ptx::mbar_init(ptx::smem_u32(&full_bar[b]), it.use_tma ? 1u : 32u * (uint32_t)it.loader_warps);
-            ptx::mbar_init(ptx::smem_u32(&empty_bar[b]), (uint32_t)units_per_item);
+            ptx::mbar_init(ptx::smem_u32(&empty_bar[b]), (uint32_t)n_compute);
         }
         abort_flag = 0;
         ptx::fence_barrier_init();
@@ -260,7 +260,8 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
         uint32_t round = 0;
         for (unsigned li = 0; li < n_local; ++li) {
             if (round > 0 && !ptx::mbar_wait_relaxed(ptx::smem_u32(&empty_bar[b]), (round - 1) & 1u, abortp)) {
-                if (!*abortp && status) atomicCAS(status, 0, kErrInputLoaderWait);
+                if (!*abortp && status) atomicCAS(status, 0, kErrInputLoaderWait | (int)(min(li, 0xFFFFu) << 8) | (int)((blockIdx.x & 0x7Fu) << 24));
+                if (status && lane == 0) { atomicCAS(status + 1, 0, (int)(0x40000000u | li | (b << 16) | (blockIdx.x << 20))); }
                 *abortp = 1;
                 break;
             }
@@ -317,59 +318,63 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
         // ------------------------------- compute -------------------------------
         const int cw = warp - it.loader_warps;
         const long long plane_bytes = (long long)g.v_plane * eb;
-        // this warp's units: cw, cw + n_compute, ... of the CTA's (item, tile[, half]) sequence, tracked incrementally
-        unsigned li = 0;
-        int within = cw, b = 0;
+        // Every compute warp waits for every item, in order, and releases it, so that no buffer can run more
+        // than one phase ahead of any warp (copies of different items may land out of order, and a parity
+        // wait cannot tell a phase that is two behind from one that is done).  Of the item's units
+        // (tile[, half]) a warp transforms those whose running index is congruent to it modulo n_compute.
+        int b = 0, start = 0;                              // start = (li * units_per_item) mod n_compute
         uint32_t round = 0;
-        for (;;) {
-            while (within >= units_per_item) {
-                within -= units_per_item;
-                ++li;
-                if (++b == it.nbuf) {
-                    b = 0;
-                    ++round;
-                }
-            }
-            if (li >= n_local) break;
-            const int t = PAIR ? within : (within >> 1), half = PAIR ? 0 : (within & 1);
+        for (unsigned li = 0; li < n_local; ++li) {
             if (!ptx::mbar_wait_relaxed(ptx::smem_u32(&full_bar[b]), round & 1u, abortp)) {
-                if (!*abortp && status) atomicCAS(status, 0, kErrInputComputeWait);
+                if (!*abortp && status)
+                    atomicCAS(status, 0, kErrInputComputeWait | (int)(min(li, 0xFFFFu) << 8) | (int)((blockIdx.x & 0x7Fu) << 24));
                 *abortp = 1;
                 break;
             }
             const int4 desc = item_desc[b];
             const int img = desc.x, ty = desc.y, tx0 = desc.z, cb = desc.w;
-            const int tx = tx0 + t;
-            const int c = cb * kItChannels + (PAIR ? 2 * lane : half * 32 + lane);
-            if (tx < g.tw && c < g.cin_pad) {
-                const long long tile = ((long long)img * g.th + ty) * g.tw + tx;
-                const int iw0 = tx0 * g.m - g.pad;
-                const int s0 = (iw0 % it.vec + it.vec) % it.vec + t * g.m;     // staged column of the tile's first input column
-                const float* p0 = s_buf + (size_t)b * it.buf_words + (size_t)(PAIR ? lane : half * 32 + lane) * it.wb + (s0 & ~3);
-                const float* p1 = p0 + 32 * it.wb;
-                T h[ALPHA][ALPHA];
-                switch (s0 & 3) {
-                    case 0: rows_pass<ALPHA, SYM, 0, T>(p0, p1, row_words, Bt, h); break;
-                    case 1: rows_pass<ALPHA, SYM, 1, T>(p0, p1, row_words, Bt, h); break;
-                    case 2: rows_pass<ALPHA, SYM, 2, T>(p0, p1, row_words, Bt, h); break;
-                    default: rows_pass<ALPHA, SYM, 3, T>(p0, p1, row_words, Bt, h); break;
-                }
-                const long long off = (tile * g.cin_pad + c) * eb;
-                char* hi = V_hi + off;
-                char* lo = V_lo ? V_lo + off : nullptr;
-                switch (mode) {
-                    case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T>(h, Bt, hi, lo, plane_bytes); break;
-                    case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T>(h, Bt, hi, lo, plane_bytes); break;
-                    case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
-                    case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
-                    default: cols_pass_store<ALPHA, SYM, STORE_FP32, T>(h, Bt, hi, lo, plane_bytes); break;
+            const int iw0 = tx0 * g.m - g.pad;
+            const int lead = (iw0 % it.vec + it.vec) % it.vec;             // staged columns ahead of the segment
+            for (int within = (cw - start + n_compute) % n_compute; within < units_per_item; within += n_compute) {
+                const int t = PAIR ? within : (within >> 1), half = PAIR ? 0 : (within & 1);
+                const int tx = tx0 + t;
+                const int c = cb * kItChannels + (PAIR ? 2 * lane : half * 32 + lane);
+                if (tx < g.tw && c < g.cin_pad) {
+                    const long long tile = ((long long)img * g.th + ty) * g.tw + tx;
+                    const int s0 = lead + t * g.m;                         // staged column of the tile's first input column
+                    const float* p0 = s_buf + (size_t)b * it.buf_words + (size_t)(PAIR ? lane : half * 32 + lane) * it.wb + (s0 & ~3);
+                    const float* p1 = p0 + 32 * it.wb;
+                    T h[ALPHA][ALPHA];
+                    switch (s0 & 3) {
+                        case 0: rows_pass<ALPHA, SYM, 0, T>(p0, p1, row_words, Bt, h); break;
+                        case 1: rows_pass<ALPHA, SYM, 1, T>(p0, p1, row_words, Bt, h); break;
+                        case 2: rows_pass<ALPHA, SYM, 2, T>(p0, p1, row_words, Bt, h); break;
+                        default: rows_pass<ALPHA, SYM, 3, T>(p0, p1, row_words, Bt, h); break;
+                    }
+                    const long long off = (tile * g.cin_pad + c) * eb;
+                    char* hi = V_hi + off;
+                    char* lo = V_lo ? V_lo + off : nullptr;
+                    switch (mode) {
+                        case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T>(h, Bt, hi, lo, plane_bytes); break;
+                        case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T>(h, Bt, hi, lo, plane_bytes); break;
+                        case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
+                        case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
+                        default: cols_pass_store<ALPHA, SYM, STORE_FP32, T>(h, Bt, hi, lo, plane_bytes); break;
+                    }
                 }
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[b]));
-            within += n_compute;
+            start += units_per_item % n_compute;
+            if (start >= n_compute) start -= n_compute;
+            if (++b == it.nbuf) {
+                b = 0;
+                ++round;
+            }
         }
     }
+    // After a wait ran out, give copies still in flight time to land before this CTA's shared memory is released.
+    if (*abortp) __nanosleep(200000);
 }
 
 // True when Bt (alpha x alpha, row-major) has the zero pattern and the +p / -p row symmetry
