@@ -49,6 +49,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const float* __restrict__ x
                                                      long long T, int mode)
 {
     __shared__ float tile[32][33];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the previous kernel of the stream has completed
     const long long t0 = (long long)blockIdx.x * 32;
     const int kk0 = blockIdx.y * 32;
     const int Kd = g.Cin * g.k * g.k;
@@ -205,8 +207,7 @@ cudaError_t launch_gather(const float* x, void* V_hi, void* V_lo, const GatherGe
     const long long bx = (T + 31) / 32;
     const int by = (g.k_pad + 31) / 32;
     if (bx > 2147483647ll || by > 65535) return cudaErrorInvalidValue;
-    gather_kernel<<<dim3((unsigned)bx, (unsigned)by), 256, 0, stream>>>(x, V_hi, V_lo, g, T, mode);
-    return cudaGetLastError();
+    return launch_overlapped(gather_kernel, dim3((unsigned)bx, (unsigned)by), dim3(256), 0, stream, x, V_hi, V_lo, g, T, mode);
 }
 
 cudaError_t launch_direct(const float* x, const float* w, const float* bias, float* y, const DirectGeom& g,

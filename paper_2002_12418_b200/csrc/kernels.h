@@ -4,7 +4,31 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace mnnb {
+
+// Launch with programmatic stream serialisation allowed: the kernel may be scheduled while the previous
+// kernel of the stream is still finishing, provided that kernel has triggered its dependents.  Every kernel
+// launched this way calls grid_dependency_wait() (umma.cuh) before it touches global memory, which blocks
+// until the previous kernel has completed and its writes are visible; so only launch latency and the
+// kernel's own set-up overlap.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 // How transformed operands are stored.
 enum StoreMode {
@@ -78,7 +102,7 @@ struct UmmaContract {
     int passes;        // 1 or 3
     int alpha2, Cout, cin_pad;
     long long tiles_capacity;
-    int bn;            // MMA N (output channels per work item), multiple of 16, <= 256
+    int bn;            // MMA N (tiles per work item), multiple of 16, <= 256
     int n_co_blocks;
     int k_blocks;
     int stages;

@@ -10,6 +10,11 @@
 namespace mnnb {
 namespace ptx {
 
+// Programmatic dependent launch: let the next kernel of the stream be scheduled / wait for the previous
+// kernel of the stream to have completed (with its writes visible).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);

@@ -248,6 +248,8 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
         if (it.use_tma) ptx::prefetch_tensormap(&xmap);
     }
     __syncthreads();
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
 
     // items of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ... (32-bit: the host keeps n_items below 2^31)
     const unsigned first = blockIdx.x, n_items = (unsigned)it.n_items;
@@ -454,9 +456,8 @@ cudaError_t launch_input_ws(const float* x, void* V_hi, void* V_lo, const WinoGe
     auto launch = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kItSmemBudget);
         if (e != cudaSuccess) return e;
-        kern<<<(unsigned)grid, kItThreads, smem, stream>>>(x, xmap, static_cast<char*>(V_hi), static_cast<char*>(V_lo), g, it,
-                                                           mode, bt, status);
-        return cudaGetLastError();
+        return launch_overlapped(kern, dim3((unsigned)grid), dim3(kItThreads), smem, stream, x, xmap, static_cast<char*>(V_hi),
+                                 static_cast<char*>(V_lo), g, it, mode, bt, status);
     };
     if (sym) return launch(input_transform_ws_kernel<ALPHA, true, kPair>);
     return launch(input_transform_ws_kernel<ALPHA, false, kPair>);

@@ -60,6 +60,8 @@ __global__ void __launch_bounds__(kOutThreads) output_transform_kernel(const flo
                                                                        const float* __restrict__ bias,
                                                                        float* __restrict__ y, WinoGeom g, int relu, MatAt At)
 {
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
     const long long tile = (long long)blockIdx.x * kOutThreads + threadIdx.x;
     const int co = blockIdx.y;
     if (tile >= g.tiles) return;
@@ -119,8 +121,7 @@ cudaError_t launch_output_am(const float* Mx, const float* bias, float* y, const
     MatAt at;
     for (int i = 0; i < M * ALPHA; ++i) at.v[i] = mats.At[i];
     dim3 grid((unsigned)((g.tiles + kOutThreads - 1) / kOutThreads), (unsigned)g.Cout);
-    output_transform_kernel<ALPHA, M><<<grid, kOutThreads, 0, stream>>>(Mx, bias, y, g, relu, at);
-    return cudaGetLastError();
+    return launch_overlapped(output_transform_kernel<ALPHA, M>, grid, dim3(kOutThreads), 0, stream, Mx, bias, y, g, relu, at);
 }
 
 
