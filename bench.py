@@ -243,6 +243,9 @@ def main():
 
     layers = workload_layers(args.workload)
     prec = B.PREC_TF32 if args.precision == "tf32" else B.PREC_BF16
+    # pre-inference: the planner's cost constants are measured once on this GPU, before any plan is made
+    calibration = B.mnn_calibrate(local_rank, torch.cuda.current_stream(dev).cuda_stream)
+    torch.cuda.synchronize(dev)
     # every rank works on its own batch of the same shape (weak scaling; images are independent)
     state = []
     for i, layer in enumerate(layers):
@@ -383,7 +386,7 @@ def main():
                 "data": "synthetic",
                 "config": {"workload": args.workload, "layers": len(layers), "batch_per_gpu": layers[0].N,
                            "l2": "flushed before every step (256 MB write)", "weights": "pre-transformed",
-                           "accuracy_class": args.precision, "plans": per_layer},
+                           "accuracy_class": args.precision, "planner_calibration": calibration[:9], "plans": per_layer},
                 "clocks": clocks, "roofline": roofline,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms / e2e_steps},

@@ -78,8 +78,10 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
  *   points_id  interpolation point set of the generator (Eq. 8): PAPER = 0, +-1/2,
  *              +-1, ... (the paper's f = 1/2); UNIT = 0, +-1, +-2, ...; MIXED = 0, +-1,
  *              +-1/2, +-2, +-1/4, +-4; AUTO = the set with the lowest predicted error.
- *   chunk_images  0 = planner; else images per pipeline chunk (the batch is cut so
- *              that the transformed tensors of one chunk stay in L2).
+ *   chunk_images  0 = planner; else images per pipeline chunk.  The planner cuts the
+ *              batch when the cost model predicts a gain from keeping one chunk's
+ *              transformed tensors in L2, and always when those tensors would exceed
+ *              4 GiB for the whole batch.
  */
 typedef struct {
     int groups;
@@ -227,7 +229,7 @@ MNN_API long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int
 /* Cost-model constants (Eq. 5's FLOPS and t_schedule, re-stated for this GPU).
  * consts[0] attoseconds per HBM byte          consts[1] attoseconds per L2-resident byte
  * consts[2] attoseconds per TF32 tensor flop  consts[3] attoseconds per BF16 tensor flop
- * consts[4] attoseconds per fp32 ALU flop     consts[5] picoseconds per kernel launch
+ * consts[4] attoseconds per fp32 ALU flop     consts[5] picoseconds of fixed cost per kernel (launch, ramp-up, tail)
  * consts[6] L2 bytes usable for one chunk     consts[7] number of SMs
  * consts[8] attoseconds per flop of the direct kernel
  * consts[9..15] reserved (0).

@@ -149,6 +149,30 @@ extern "C" int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CO
         cal.c[2 + kind] = to_ll(t * 1e15 / flops);
     }
 
+    // fixed cost of one kernel of the pipeline (launch, ramp-up, tail): the contraction on a problem of four work items
+    {
+        const int alpha2 = 4, Cout = 128, cin = 64;
+        const long long tiles = 128;
+        char* U = buf + 1024;
+        char* V = U + (1 << 20);
+        char* M = V + (1 << 20);
+        cudaMemsetAsync(buf, 0, 1024, st);
+        UmmaContract uc;
+        const char* why = "";
+        if (umma_contract_setup(&uc, STORE_BF16, alpha2, Cout, cin, tiles, U, nullptr, V, nullptr, &why) == cudaSuccess) {
+            ContractEpilogue epi = {0, reinterpret_cast<float*>(M), tiles, nullptr, nullptr, 0, 1};
+            int* status = reinterpret_cast<int*>(buf);
+            for (int i = 0; i < 5; ++i) launch_contract_umma(uc, tiles, epi, status, st);
+            tm.start();
+            const int reps = 50;
+            for (int i = 0; i < reps; ++i) launch_contract_umma(uc, tiles, epi, status, st);
+            ms = tm.stop();
+            int code = 0;
+            cudaMemcpy(&code, status, sizeof(int), cudaMemcpyDeviceToHost);
+            if (code == 0 && ms > 0.0) cal.c[5] = to_ll(ms / reps * 1e9);
+        }
+    }
+
     // direct kernel rate: 3x3, 64 -> 64 channels, 56 x 56, 4 images
     {
         DirectGeom g = {4, 64, 64, 56, 56, 56, 56, 3, 1, 1, 1, 1, 1};

@@ -27,6 +27,7 @@ Calibration g_cal;
 bool g_cal_set = false;
 
 uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+constexpr uint64_t kMaxChunkBytes = 4ull << 30;   // V + M of one chunk
 uint64_t round_up(uint64_t a, uint64_t b) { return ceil_div(a, b) * b; }
 uint64_t max3(uint64_t a, uint64_t b, uint64_t c) { return a > b ? (a > c ? a : c) : (b > c ? b : c); }
 }  // namespace
@@ -35,15 +36,16 @@ Calibration default_calibration()
 {
     Calibration c;
     std::memset(&c, 0, sizeof(c));
-    c.c[0] = 160000;      // as per HBM byte          (~6.2 TB/s)
-    c.c[1] = 70000;       // as per L2-resident byte  (~14 TB/s)
-    c.c[2] = 2000;        // as per TF32 tensor flop  (~500 TFLOP/s achieved)
-    c.c[3] = 1000;        // as per BF16 tensor flop  (~1000 TFLOP/s achieved)
+    // one calibration record measured on a B200 (mnn_calibrate), rounded
+    c.c[0] = 171000;      // as per HBM byte          (~5.8 TB/s with a plain copy kernel)
+    c.c[1] = 75000;       // as per L2-resident byte  (~13 TB/s)
+    c.c[2] = 2440;        // as per TF32 tensor flop  (~410 TFLOP/s achieved by the contraction kernel)
+    c.c[3] = 1390;        // as per BF16 tensor flop  (~720 TFLOP/s achieved)
     c.c[4] = 28000;       // as per fp32 ALU flop in the transform kernels (~36 TFLOP/s)
-    c.c[5] = 2500000;     // ps per kernel launch (the t_schedule of Eq. 5)
+    c.c[5] = 5500000;     // ps of fixed cost per kernel: launch, ramp-up and tail (the t_schedule of Eq. 5)
     c.c[6] = 80ll << 20;  // L2 bytes one chunk's V + M may occupy
     c.c[7] = 148;         // SMs
-    c.c[8] = 100000;      // as per flop of the direct kernel (~10 TFLOP/s)
+    c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
     return c;
 }
 
@@ -324,7 +326,9 @@ uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes
     const uint64_t y_bytes = 4ull * n * s.Cout * s.OH * s.OW;
     const uint64_t cV = (uint64_t)(resident ? cal.c[1] : cal.c[0]);
     const uint64_t c0 = (uint64_t)cal.c[0], cA = (uint64_t)cal.c[4];
-    const uint64_t in = kernel_ps(x_bytes * c0 + v_bytes * cV, 0, 4ull * alpha * a2 * n * tiles_img * s.Cin * cA, cal);
+    // from alpha = 8 on a lane of the input transform holds one channel instead of a packed pair: twice the ALU time
+    const uint64_t in_alu = (alpha >= 8 ? 2ull : 1ull) * 4ull * alpha * a2 * n * tiles_img * s.Cin * cA;
+    const uint64_t in = kernel_ps(x_bytes * c0 + v_bytes * cV, 0, in_alu, cal);
     const uint64_t con = kernel_ps((v_bytes + m_bytes) * cV + u_bytes * c0,
                                    2ull * a2 * s.Cout * Cp * n * tiles_img * passes * tensor_as(operand, cal), 0, cal);
     const uint64_t out = kernel_ps(m_bytes * cV + y_bytes * c0, 0,
@@ -344,12 +348,17 @@ void winograd_chunking(const LayerShape& s, int m, int operand, int passes, cons
     const uint64_t per_img = a2 * tiles_img * Cp * b_el + a2 * (uint64_t)s.Cout * tiles_img * 4;
     const uint64_t N = (uint64_t)s.N;
     const uint64_t n_fit = per_img ? (uint64_t)cal.c[6] / per_img : N;
+    // the transformed tensors of one chunk may not exceed kMaxChunkBytes, whatever the cost says
+    uint64_t n_cap = per_img ? kMaxChunkBytes / per_img : N;
+    if (n_cap < 1) n_cap = 1;
 
-    // option A: the whole batch in one chunk
-    const uint64_t costA = winograd_chunk_cost(s, m, operand, passes, N, n_fit >= N, cal);
+    // option A: the largest chunk the cap allows (the whole batch if it fits)
+    const uint64_t chunkA = N < n_cap ? N : ceil_div(N, ceil_div(N, n_cap));
+    const uint64_t nA = ceil_div(N, chunkA);
+    const uint64_t costA = nA * winograd_chunk_cost(s, m, operand, passes, chunkA, n_fit >= chunkA, cal);
     uint64_t best_cost = costA;
-    uint64_t best_chunk = N, best_n = 1;
-    if (n_fit >= 1 && n_fit < N) {
+    uint64_t best_chunk = chunkA, best_n = nA;
+    if (n_fit >= 1 && n_fit < chunkA) {
         // option B: chunks whose V + M stay in L2
         const uint64_t nch = ceil_div(N, n_fit);
         const uint64_t chunk = ceil_div(N, nch);

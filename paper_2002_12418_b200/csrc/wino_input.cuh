@@ -9,7 +9,7 @@
 // columns; or two boxes of 32 channels, even and odd, through a 5-D view of x that splits
 // the channel parity); everything outside the image, including the zero padding of the
 // convolution and channels beyond Cin, arrives as zeros, so several items are in flight
-// with no load instructions at all.  Otherwise four loader warps issue contiguous cp.async
+// with no load instructions at all.  Otherwise eight loader warps issue contiguous cp.async
 // copies with explicit zero fill.  The remaining warps take (item, tile) units in order.  A
 // lane transforms one tile of TWO adjacent channels held as packed fp32 pairs (packed
 // fp32x2 multiply-adds), or of one channel for alpha >= 8 where a pair would not fit the
@@ -40,6 +40,7 @@ constexpr int kItChannels = 64;         // channels per work item
 constexpr int kItWarps = 16;
 constexpr int kItThreads = 32 * kItWarps;
 constexpr int kItMaxBuffers = 6;
+constexpr int kItCopySlots = 12;        // cp.async path: at most 32 * 12 copies per channel of an item
 constexpr int kItSmemBudget = 200 * 1024;
 constexpr int kErrInputLoaderWait = 11, kErrInputComputeWait = 12;
 
@@ -53,7 +54,7 @@ struct InputItems {
     int cblocks;        // blocks of 64 channels
     int use_tma;        // 1: TMA box copies (W % 4 == 0), 0: cp.async
     int vec;            // alignment of the staged column grid in elements: 4 with TMA, else 2 or 1
-    int loader_warps;   // 1 with TMA, else 4
+    int loader_warps;   // 1 with TMA, else 8
     int buf_words;      // words per buffer = alpha * 64 * wb
     long long n_items;
 };
@@ -260,6 +261,17 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
         // ------------------------------- loaders -------------------------------
         int b = 0;
         uint32_t round = 0;
+        int copy_r[kItCopySlots], copy_j[kItCopySlots];       // cp.async path: this lane's (row, first column) per step
+        {
+            const int per_row = it.wb / it.vec;
+#pragma unroll
+            for (int i = 0; i < kItCopySlots; ++i) {
+                const int e = lane + 32 * i;
+                const int r = e / per_row;
+                copy_r[i] = (!it.use_tma && r < ALPHA) ? r : -1;
+                copy_j[i] = (e - r * per_row) * it.vec;
+            }
+        }
         for (unsigned li = 0; li < n_local; ++li) {
             if (round > 0 && !ptx::mbar_wait_relaxed(ptx::smem_u32(&empty_bar[b]), (round - 1) & 1u, abortp)) {
                 if (!*abortp && status) atomicCAS(status, 0, kErrInputLoaderWait | (int)(min(li, 0xFFFFu) << 8) | (int)((blockIdx.x & 0x7Fu) << 24));
@@ -293,20 +305,30 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
                     if (lane < ALPHA) ptx::tma_load_4d(sbuf + (uint32_t)(lane * row_words) * 4u, &xmap, bar, a0, ih0 + lane, c0, img);
                 }
             } else {
-                // contiguous copies: consecutive lanes take consecutive staged elements of one (channel, row)
+                // contiguous copies: consecutive lanes take consecutive staged elements of one channel (rows of wb
+                // columns, alpha rows).  A lane's elements have the same (row, column) in every channel and item,
+                // so they are decoded once (copy_r / copy_j, before the item loop).
                 const float* ximg = x + (size_t)img * g.Cin * g.H * g.W;
-                const int per_row = it.wb / it.vec;                        // copies per staged row
-                const int per_ch = ALPHA * per_row;
-                const int total = kItChannels * per_ch;
-                for (int e = warp * 32 + lane; e < total; e += 32 * it.loader_warps) {
-                    const int c = e / per_ch, rem = e - c * per_ch;
-                    const int r = rem / per_row, jv = rem - r * per_row;
-                    const int ih = ih0 + r, iw = a0 + jv * it.vec, ci = c0 + c;
-                    const uint32_t dst = sbuf + (uint32_t)(r * row_words + slot_of<PAIR>(c) * it.wb + jv * it.vec) * 4u;
-                    const bool ok = ih >= 0 && ih < g.H && ci < g.Cin && iw >= 0 && iw + it.vec <= g.W;
-                    const float* src = ok ? ximg + ((size_t)ci * g.H + ih) * g.W + iw : ximg;
-                    if (it.vec == 2) ptx::cp_async_8(dst, src, ok ? 8u : 0u);
-                    else ptx::cp_async_4(dst, src, ok ? 4u : 0u);
+                uint32_t nbytes[kItCopySlots];
+#pragma unroll
+                for (int i = 0; i < kItCopySlots; ++i) {
+                    const int ih = ih0 + copy_r[i], iw = a0 + copy_j[i];
+                    nbytes[i] = (copy_r[i] >= 0 && ih >= 0 && ih < g.H && iw >= 0 && iw + it.vec <= g.W) ? 4u * (uint32_t)it.vec : 0u;
+                }
+                for (int c = warp; c < kItChannels; c += it.loader_warps) {
+                    const int ci = c0 + c;
+                    const bool c_ok = ci < g.Cin;
+                    const float* src = ximg + ((size_t)(c_ok ? ci : 0) * g.H + ih0) * g.W + a0;
+                    const uint32_t dst = sbuf + (uint32_t)(slot_of<PAIR>(c) * it.wb) * 4u;
+#pragma unroll
+                    for (int i = 0; i < kItCopySlots; ++i) {
+                        if (copy_r[i] < 0) break;
+                        const uint32_t nb = c_ok ? nbytes[i] : 0u;
+                        const uint32_t d = dst + (uint32_t)(copy_r[i] * row_words + copy_j[i]) * 4u;
+                        const float* sp = nb ? src + copy_r[i] * g.W + copy_j[i] : ximg;
+                        if (it.vec == 2) ptx::cp_async_8(d, sp, nb);
+                        else ptx::cp_async_4(d, sp, nb);
+                    }
                 }
                 ptx::cp_async_arrive_noinc(bar);
             }
@@ -403,7 +425,7 @@ inline bool plan_input_items(const WinoGeom& g, int alpha, bool tma_ok, InputIte
 {
     it->use_tma = tma_ok ? 1 : 0;
     it->vec = tma_ok ? 4 : ((g.W % 2 == 0) ? 2 : 1);
-    it->loader_warps = tma_ok ? 1 : 4;
+    it->loader_warps = tma_ok ? 1 : 8;
     it->cblocks = (g.cin_pad + kItChannels - 1) / kItChannels;
     for (int nseg = 1; nseg <= g.tw; ++nseg) {
         const int txs = (g.tw + nseg - 1) / nseg;
@@ -413,10 +435,12 @@ inline bool plan_input_items(const WinoGeom& g, int alpha, bool tma_ok, InputIte
         int wb = (span + (it->vec - 1) + 3 + 3) / 4 * 4;
         if (((wb / 4) & 1) == 0) wb += 4;
         if (wb > 256) continue;
+        if (!tma_ok && alpha * (wb / it->vec) > 32 * kItCopySlots && txs > 1) continue;
         const long long bytes = (long long)alpha * kItChannels * wb * 4;
         long long nbuf = kItSmemBudget / bytes;
         if (nbuf >= 3 || txs == 1) {
             if (nbuf < 2) return false;
+            if (!tma_ok && alpha * (wb / it->vec) > 32 * kItCopySlots) return false;
             if (nbuf > kItMaxBuffers) nbuf = kItMaxBuffers;
             it->txs = txs;
             it->nseg = (g.tw + txs - 1) / txs;
