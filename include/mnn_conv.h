@@ -79,9 +79,8 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
  *              +-1, ... (the paper's f = 1/2); UNIT = 0, +-1, +-2, ...; MIXED = 0, +-1,
  *              +-1/2, +-2, +-1/4, +-4; AUTO = the set with the lowest predicted error.
  *   chunk_images  0 = planner; else images per pipeline chunk.  The planner cuts the
- *              batch when the cost model predicts a gain from keeping one chunk's
- *              transformed tensors in L2, and always when those tensors would exceed
- *              4 GiB for the whole batch.
+ *              batch only when the transformed tensors of the whole batch would
+ *              exceed 4 GiB.
  */
 typedef struct {
     int groups;

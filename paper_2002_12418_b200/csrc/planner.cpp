@@ -358,17 +358,9 @@ void winograd_chunking(const LayerShape& s, int m, int operand, int passes, cons
     const uint64_t costA = nA * winograd_chunk_cost(s, m, operand, passes, chunkA, n_fit >= chunkA, cal);
     uint64_t best_cost = costA;
     uint64_t best_chunk = chunkA, best_n = nA;
-    if (n_fit >= 1 && n_fit < chunkA) {
-        // option B: chunks whose V + M stay in L2
-        const uint64_t nch = ceil_div(N, n_fit);
-        const uint64_t chunk = ceil_div(N, nch);
-        const uint64_t costB = nch * winograd_chunk_cost(s, m, operand, passes, chunk, true, cal);
-        if (costB <= costA) {
-            best_cost = costB;
-            best_chunk = chunk;
-            best_n = ceil_div(N, chunk);
-        }
-    }
+    // Cutting the batch further so that a chunk's V and M stay in L2 was measured on B200 and never paid:
+    // the fixed cost of three more kernels per chunk outweighs what the kernels gain from L2-resident
+    // operands.  The L2 rate is still used for the byte cost when a whole chunk fits.
     *chunk_images = (int)best_chunk;
     *n_chunks = (int)best_n;
     *cost_ps = best_cost;
