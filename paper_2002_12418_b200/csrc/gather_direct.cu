@@ -118,20 +118,25 @@ __global__ void __launch_bounds__(256) direct_generic_kernel(const float* __rest
     }
 }
 
-// Depthwise 3x3 (groups = C, dilation 1, stride 1 or 2): one warp sweeps a 32-column
-// strip of one channel plane downwards.  Each lane keeps the three input rows of its
-// output column group in registers; horizontal neighbours come from warp shuffles, so
-// every input element is loaded once per strip.
+// Depthwise 3x3 (groups = C, dilation 1, padding 1, stride 1 or 2): one warp sweeps a strip of one channel
+// plane downwards over a band of output rows.  A lane holds its column of the three input rows that an output
+// row needs; horizontal neighbours come from warp shuffles, so every input element is loaded once per strip
+// (plus two halo rows per band).  Four input rows are requested before any of them is used, which keeps
+// enough loads in flight for the kernel to follow the memory system rather than its latency.
+constexpr int kDwBandRows = 32;   // output rows per unit
+
 template <int STRIDE>
 __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restrict__ x, const float* __restrict__ w,
                                                            const float* __restrict__ bias, float* __restrict__ y,
-                                                           DirectGeom g, int strips, long long n_units)
+                                                           DirectGeom g, int strips, int bands, long long n_units)
 {
     const int lane = threadIdx.x & 31;
-    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (plane, strip)
+    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (plane, band, strip)
     if (unit >= n_units) return;
-    const long long plane = unit / strips;
     const int strip = (int)(unit % strips);
+    const long long rest = unit / strips;
+    const int band = (int)(rest % bands);
+    const long long plane = rest / bands;
     const int c = (int)(plane % g.Cout);
     const float* xp = x + (size_t)plane * g.H * g.W;
     float* yp = y + (size_t)plane * g.OH * g.OW;
@@ -139,61 +144,78 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
 #pragma unroll
     for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + (size_t)c * 9 + i);
     const float b = bias ? __ldg(bias + c) : 0.0f;
+    const int oh0 = band * kDwBandRows, oh1 = min(g.OH, oh0 + kDwBandRows);
+    const unsigned full = 0xffffffffu;
 
-    // Lane l produces output column ow = strip*30 + l - 1 + ... for stride 1 we let the 32 lanes
-    // hold 32 input columns iw0 + l and produce outputs from the 30 interior lanes.
     if (STRIDE == 1) {
-        const int iw = strip * 30 - g.pad + lane;           // input column held by this lane
-        const int ow = iw - 1 + g.pad;                      // output whose centre tap is this column (pad = 1 -> ow = iw)
+        // the 32 lanes hold input columns strip * 30 - 1 + lane; the 30 interior lanes produce outputs
+        const int iw = strip * 30 - 1 + lane;
+        const int ow = iw;
         const bool col_ok = iw >= 0 && iw < g.W;
-        const bool out_ok = lane >= 1 && lane <= 30 && ow >= 0 && ow < g.OW;
-        float r0 = 0.0f, r1 = 0.0f, r2;
-        // rows: output row oh uses input rows oh - pad + {0,1,2}
-        int ih = -g.pad;
-        r0 = (col_ok && ih >= 0 && ih < g.H) ? __ldg(xp + (size_t)ih * g.W + iw) : 0.0f;
-        ++ih;
-        r1 = (col_ok && ih >= 0 && ih < g.H) ? __ldg(xp + (size_t)ih * g.W + iw) : 0.0f;
-        for (int oh = 0; oh < g.OH; ++oh) {
-            ih = oh - g.pad + 2;
-            r2 = (col_ok && ih >= 0 && ih < g.H) ? __ldg(xp + (size_t)ih * g.W + iw) : 0.0f;
-            float acc = b;
-            const float l0 = __shfl_up_sync(0xffffffffu, r0, 1), l1 = __shfl_up_sync(0xffffffffu, r1, 1),
-                        l2 = __shfl_up_sync(0xffffffffu, r2, 1);
-            const float q0 = __shfl_down_sync(0xffffffffu, r0, 1), q1 = __shfl_down_sync(0xffffffffu, r1, 1),
-                        q2 = __shfl_down_sync(0xffffffffu, r2, 1);
-            acc = fmaf(wk[0], l0, acc); acc = fmaf(wk[1], r0, acc); acc = fmaf(wk[2], q0, acc);
-            acc = fmaf(wk[3], l1, acc); acc = fmaf(wk[4], r1, acc); acc = fmaf(wk[5], q1, acc);
-            acc = fmaf(wk[6], l2, acc); acc = fmaf(wk[7], r2, acc); acc = fmaf(wk[8], q2, acc);
-            if (out_ok) yp[(size_t)oh * g.OW + ow] = g.relu ? fmaxf(acc, 0.0f) : acc;
-            r0 = r1;
-            r1 = r2;
+        const bool out_ok = lane >= 1 && lane <= 30 && ow < g.OW;
+        auto row = [&](int ih) { return (col_ok && ih >= 0 && ih < g.H) ? __ldg(xp + (size_t)ih * g.W + iw) : 0.0f; };
+        // per input row: the lane's own value and its left / right neighbours (shuffled once, when the row arrives)
+        float r0 = row(oh0 - 1), r1 = row(oh0);
+        float l0 = __shfl_up_sync(full, r0, 1), q0 = __shfl_down_sync(full, r0, 1);
+        float l1 = __shfl_up_sync(full, r1, 1), q1 = __shfl_down_sync(full, r1, 1);
+        for (int oh = oh0; oh < oh1; oh += 4) {
+            float nx[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) nx[k] = row(oh + k + 1);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (oh + k < oh1) {
+                    const float r2 = nx[k];
+                    const float l2 = __shfl_up_sync(full, r2, 1), q2 = __shfl_down_sync(full, r2, 1);
+                    float acc = b;
+                    acc = fmaf(wk[0], l0, acc); acc = fmaf(wk[1], r0, acc); acc = fmaf(wk[2], q0, acc);
+                    acc = fmaf(wk[3], l1, acc); acc = fmaf(wk[4], r1, acc); acc = fmaf(wk[5], q1, acc);
+                    acc = fmaf(wk[6], l2, acc); acc = fmaf(wk[7], r2, acc); acc = fmaf(wk[8], q2, acc);
+                    if (out_ok) yp[(size_t)(oh + k) * g.OW + ow] = g.relu ? fmaxf(acc, 0.0f) : acc;
+                    l0 = l1; r0 = r1; q0 = q1;
+                    l1 = l2; r1 = r2; q1 = q2;
+                }
+            }
         }
     } else {
-        // stride 2: lane l produces output column ow = strip*32 + l and needs input columns 2*ow - pad + {0,1,2};
-        // it loads the pair (2*ow - pad, 2*ow - pad + 1) and takes the third from the next lane.
+        // lane l produces output column ow = strip * 32 + l from input columns 2 ow - 1 + {0, 1, 2}: it loads the
+        // first two and takes the third from the next lane (the last lane loads its own)
         const int ow = strip * 32 + lane;
-        const int iw0 = 2 * ow - g.pad;
+        const int iw0 = 2 * ow - 1;
         const bool out_ok = ow < g.OW;
-        const bool c0_ok = iw0 >= 0 && iw0 < g.W, c1_ok = iw0 + 1 >= 0 && iw0 + 1 < g.W;
-        // the last lane has no right neighbour: it loads its third column itself
-        const int iw2 = iw0 + 2;
-        const bool c2_ok = iw2 >= 0 && iw2 < g.W;
-        for (int oh = 0; oh < g.OH; ++oh) {
+        const bool c0_ok = iw0 >= 0 && iw0 < g.W, c1_ok = iw0 + 1 < g.W, c2_ok = lane == 31 && iw0 + 2 < g.W;
+        struct Row { float v0, v1, v2; };
+        auto load = [&](int ih, Row& r) {
+            const bool ok = ih >= 0 && ih < g.H;
+            const float* p = xp + (size_t)(ok ? ih : 0) * g.W + iw0;
+            r.v0 = (ok && c0_ok) ? __ldg(p) : 0.0f;
+            r.v1 = (ok && c1_ok) ? __ldg(p + 1) : 0.0f;
+            r.v2 = (ok && c2_ok) ? __ldg(p + 2) : 0.0f;
+        };
+        auto third = [&](Row& r) {
+            const float n = __shfl_down_sync(full, r.v0, 1);
+            if (lane != 31) r.v2 = n;
+        };
+        auto out = [&](int oh, const Row& a, const Row& m, const Row& z) {
             float acc = b;
-#pragma unroll
-            for (int a = 0; a < 3; ++a) {
-                const int ih = 2 * oh - g.pad + a;
-                const bool row_ok = ih >= 0 && ih < g.H;
-                const float* rowp = xp + (size_t)(row_ok ? ih : 0) * g.W;
-                const float v0 = (row_ok && c0_ok) ? __ldg(rowp + iw0) : 0.0f;
-                const float v1 = (row_ok && c1_ok) ? __ldg(rowp + iw0 + 1) : 0.0f;
-                float v2 = __shfl_down_sync(0xffffffffu, v0, 1);
-                if (lane == 31) v2 = (row_ok && c2_ok) ? __ldg(rowp + iw2) : 0.0f;
-                acc = fmaf(wk[a * 3 + 0], v0, acc);
-                acc = fmaf(wk[a * 3 + 1], v1, acc);
-                acc = fmaf(wk[a * 3 + 2], v2, acc);
-            }
+            acc = fmaf(wk[0], a.v0, acc); acc = fmaf(wk[1], a.v1, acc); acc = fmaf(wk[2], a.v2, acc);
+            acc = fmaf(wk[3], m.v0, acc); acc = fmaf(wk[4], m.v1, acc); acc = fmaf(wk[5], m.v2, acc);
+            acc = fmaf(wk[6], z.v0, acc); acc = fmaf(wk[7], z.v1, acc); acc = fmaf(wk[8], z.v2, acc);
             if (out_ok) yp[(size_t)oh * g.OW + ow] = g.relu ? fmaxf(acc, 0.0f) : acc;
+        };
+        Row prev;
+        load(2 * oh0 - 1, prev);
+        third(prev);
+        for (int oh = oh0; oh < oh1; oh += 2) {
+            Row ra, rb, rc, rd;                       // input rows 2 oh .. 2 oh + 3, all requested before use
+            load(2 * oh, ra);
+            load(2 * oh + 1, rb);
+            load(2 * oh + 2, rc);
+            load(2 * oh + 3, rd);
+            third(ra); third(rb); third(rc); third(rd);
+            out(oh, prev, ra, rb);
+            if (oh + 1 < oh1) out(oh + 1, rb, rc, rd);
+            prev = rd;
         }
     }
 }
@@ -220,13 +242,14 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
     if (depthwise3) {
         const long long planes = (long long)g.N * g.Cout;
         const int strips = g.stride == 1 ? (g.OW + 29) / 30 : (g.OW + 31) / 32;
-        const long long units = planes * strips;
+        const int bands = (g.OH + kDwBandRows - 1) / kDwBandRows;
+        const long long units = planes * strips * bands;
         const long long blocks = (units + 3) / 4;
         if (blocks > 2147483647ll) return cudaErrorInvalidValue;
         if (g.stride == 1)
-            depthwise3x3_kernel<1><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, units);
+            depthwise3x3_kernel<1><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, units);
         else
-            depthwise3x3_kernel<2><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, units);
+            depthwise3x3_kernel<2><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, units);
         return cudaGetLastError();
     }
     long long blocks = (total + 255) / 256;
