@@ -3,15 +3,17 @@
 // per transform position xi):
 //     out[xi][co][t] = sum_c U[xi][co][c] * V[xi][t][c]
 // A persistent, warp-specialised kernel: one thread feeds shared memory with TMA
-// (128-byte-swizzled K-major tiles of U and V), one thread issues tcgen05.mma with
-// the accumulator in tensor memory (128 output channels x BN tiles, double
+// (128-byte-swizzled K-major tiles of V and U), one thread issues tcgen05.mma with
+// the accumulator in tensor memory (128 tiles x BN output channels, double
 // buffered), four warps drain the accumulator with tcgen05.ld and store it.
-// The MMA "M" dimension is the output channel (operand A = U), "N" the tile index
-// (operand B = V), "K" the input channel; TF32 or BF16 operands, fp32 accumulation;
+// The MMA "M" dimension is the tile index t (operand A = V), "N" the output channel
+// (operand B = U), "K" the input channel; TF32 or BF16 operands, fp32 accumulation;
 // with passes = 3 the operands come as hi + lo pairs and hi*hi + lo*hi + hi*lo are
-// accumulated.  In tensor memory a lane is an output channel and a column a tile, so an
-// epilogue thread holds 16 consecutive tiles of one channel: 64 contiguous bytes of
-// out[xi][co][.], written with 128-bit stores.
+// accumulated.  In tensor memory a lane is a tile and a column an output channel, so
+// the 32 lanes of an epilogue warp write 128 contiguous bytes of out[xi][co][.] per
+// store: one full line per request.  (With channels on the lanes and 128-bit stores
+// the instruction count is lower but every store touches 32 rows; measured slower on
+// short K loops, where the epilogue decides.)
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -22,13 +24,14 @@ namespace mnnb {
 namespace {
 
 constexpr int kThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
-constexpr int kTileM = 128;            // output channels (rows of U) per work item
+constexpr int kTileM = 128;            // tiles (rows of V) per work item
 constexpr int kMaxStages = 8;
+constexpr int kMaxSharedBias = 2048;    // output channels whose bias is staged in shared memory
 constexpr int kSwizzleBytes = 128;     // bytes of K per shared-memory row
 constexpr int kSmemBudget = 200 * 1024;
 
 struct KernelParams {
-    int alpha2, n_tile_blocks, n_co_blocks, bn, k_blocks, passes, stages, tmem_cols;   // bn = tiles per work item
+    int alpha2, n_tile_blocks, n_co_blocks, bn, k_blocks, passes, stages, tmem_cols;   // bn = output channels per work item
     int Cout;
     long long tiles;
     long long n_items;
@@ -52,11 +55,12 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     __shared__ __align__(8) uint64_t tempty_bar[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ __align__(16) float s_bias[kMaxSharedBias];   // GEMM scheme: bias (zeros if none) for the epilogue
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = kTileM * kSwizzleBytes;                 // one U tile (128 output channels)
-    const uint32_t b_bytes = (uint32_t)p.bn * kSwizzleBytes;         // one V tile (bn tiles)
+    const uint32_t a_bytes = kTileM * kSwizzleBytes;                 // one V tile (128 tiles)
+    const uint32_t b_bytes = (uint32_t)p.bn * kSwizzleBytes;         // one U tile (bn output channels)
     const uint32_t split = p.passes == 3 ? 2u : 1u;
     const uint32_t stage_bytes = (a_bytes + b_bytes) * split;
     // stage layout: [A_hi][A_lo?][B_hi][B_lo?]
@@ -87,6 +91,11 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     const uint32_t tmem_base = tmem_slot;
     ptx::grid_launch_dependents();
     ptx::grid_dependency_wait();
+    const bool bias_in_smem = p.epi.mode == 1 && p.Cout <= kMaxSharedBias;
+    if (bias_in_smem && warp >= 2) {
+        for (int i = threadIdx.x - 64; i < p.Cout; i += kThreads - 64) s_bias[i] = p.epi.bias ? __ldg(p.epi.bias + i) : 0.0f;
+        asm volatile("bar.sync 1, 128;" ::: "memory");          // the four epilogue warps only
+    }
 
     const int k_elems = KIND == 0 ? 32 : 64;         // elements of K per 128-byte row
 
@@ -109,11 +118,11 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
                     const uint32_t sbase = smem_base + stage * stage_bytes;
                     ptx::mbar_expect_tx(bar, stage_bytes);
-                    ptx::tma_load_3d(sbase, &map_u_hi, bar, kb * k_elems, nb * kTileM, xi);
-                    ptx::tma_load_3d(sbase + off_b_hi, &map_v_hi, bar, kb * k_elems, tb * p.bn, xi);
+                    ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
+                    ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
                     if (split == 2) {
-                        ptx::tma_load_3d(sbase + off_a_lo, &map_u_lo, bar, kb * k_elems, nb * kTileM, xi);
-                        ptx::tma_load_3d(sbase + off_b_lo, &map_v_lo, bar, kb * k_elems, tb * p.bn, xi);
+                        ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM, xi);
+                        ptx::tma_load_3d(sbase + off_b_lo, &map_u_lo, bar, kb * k_elems, nb * p.bn, xi);
                     }
                     if (++stage == (uint32_t)p.stages) {
                         stage = 0;
@@ -191,55 +200,50 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 break;
             }
             ptx::tc_fence_after();
-            const int co = nb * kTileM + q * 32 + lane;           // this thread's output channel
-            const bool co_ok = co < p.Cout;
-            const long long t0 = (long long)tb * p.bn;            // first tile of the item
+            const long long t = (long long)tb * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
+            const bool t_ok = t < p.tiles;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)p.bn;
-            float* out_row = nullptr;
-            float bias = 0.0f;
+            const int co0 = nb * p.bn;
+            const int n_co = min(p.bn, p.Cout - co0);                        // valid output channels of this item
+            // destination of channel co0 for this thread, and the distance to the next channel
+            float* dst;
+            long long step;
             if (p.epi.mode == 0) {
-                out_row = p.epi.M + ((size_t)xi * p.Cout + (co_ok ? co : 0)) * p.epi.m_row_stride + t0;
-            } else if (co_ok && p.epi.bias) {
-                bias = __ldg(p.epi.bias + co);
+                step = p.epi.m_row_stride;
+                dst = p.epi.M + ((size_t)xi * p.Cout + co0) * p.epi.m_row_stride + t;
+            } else {
+                const long long img = t_ok ? t / p.epi.ohw : 0;
+                step = p.epi.ohw;
+                dst = p.epi.y + ((size_t)img * p.Cout + co0) * p.epi.ohw + (t_ok ? t - img * p.epi.ohw : 0);
             }
-            for (int c0 = 0; c0 < p.bn; c0 += 16) {
-                if (t0 + c0 >= p.tiles) break;                    // nothing but padding from here on (uniform)
+            for (int c0 = 0; c0 < n_co; c0 += 16) {
                 uint32_t v[16];
                 ptx::tmem_ld16(taddr + (uint32_t)c0, v);
                 ptx::tmem_ld_wait();
-                if (!co_ok) continue;
-                if (p.epi.mode == 0) {
-                    // rows of M are padded to a multiple of 32 tiles: whole vectors may be written
-                    float4* dst = reinterpret_cast<float4*>(out_row + c0);
+                if (t_ok) {
+                    const int n = min(16, n_co - c0);
+                    if (p.epi.mode == 0) {
+                        if (n == 16) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                } else {
-                    const long long t = t0 + c0;
-                    const long long img = t / p.epi.ohw;
-                    const int pix = (int)(t - img * p.epi.ohw);
-                    float o[16];
+                            for (int j = 0; j < 16; ++j) dst[(long long)j * step] = __uint_as_float(v[j]);
+                        } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        o[j] = __uint_as_float(v[j]) + bias;
-                        if (p.epi.relu) o[j] = fmaxf(o[j], 0.0f);
-                    }
-                    if ((p.epi.ohw & 3) == 0 && pix + 16 <= p.epi.ohw && t + 16 <= p.tiles) {
-                        float4* dst = reinterpret_cast<float4*>(p.epi.y + ((size_t)img * p.Cout + co) * p.epi.ohw + pix);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                            for (int j = 0; j < 16; ++j)
+                                if (j < n) dst[(long long)j * step] = __uint_as_float(v[j]);
+                        }
                     } else {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            const long long tj = t + j;
-                            if (tj < p.tiles) {
-                                const long long ij = tj / p.epi.ohw;
-                                p.epi.y[((size_t)ij * p.Cout + co) * p.epi.ohw + (tj - ij * p.epi.ohw)] = o[j];
+                            if (j < n) {
+                                float o = __uint_as_float(v[j]) + (bias_in_smem ? s_bias[co0 + c0 + j]
+                                                                                : (p.epi.bias ? __ldg(p.epi.bias + co0 + c0 + j) : 0.0f));
+                                if (p.epi.relu) o = fmaxf(o, 0.0f);
+                                dst[(long long)j * step] = o;
                             }
                         }
                     }
                 }
+                dst += 16 * step;
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -350,16 +354,11 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
         *why = "operand rows must be a multiple of 16 bytes";
         return cudaErrorInvalidValue;
     }
-    // tiles per work item (MMA N): 256, except for hi + lo pairs with a short K loop, where 128 leaves room
-    // for a third pipeline stage (latency matters more than operand re-use there); no more than the plan's
-    // tiles rounded up to 16
-    uc->n_co_blocks = (Cout + kTileM - 1) / kTileM;
+    // output channels per work item (MMA N): as many as fit (<= 256), multiple of 16, blocks balanced
     {
-        long long cap16 = (tiles_capacity + 15) / 16 * 16;
-        const int k_blocks_est = (cin_pad * eb + kSwizzleBytes - 1) / kSwizzleBytes;
-        int bn_max = (store_is_split(mode) && k_blocks_est < 4) ? 128 : 256;
-        uc->bn = (int)(cap16 < bn_max ? cap16 : bn_max);
-        if (uc->bn < 16) uc->bn = 16;
+        const int co16 = (Cout + 15) / 16 * 16;
+        uc->n_co_blocks = (co16 + 255) / 256;
+        uc->bn = ((co16 / 16 + uc->n_co_blocks - 1) / uc->n_co_blocks) * 16;
     }
     const int k_elems = kSwizzleBytes / eb;
     uc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
@@ -386,11 +385,11 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     if (e != cudaSuccess) return e;
 
     const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
-    bool ok = encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, uc->bn) &&
-              encode_operand_map(&uc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, kTileM);
+    bool ok = encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
+              encode_operand_map(&uc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
     if (ok && split == 2)
-        ok = encode_operand_map(&uc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, uc->bn) &&
-             encode_operand_map(&uc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, kTileM);
+        ok = encode_operand_map(&uc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
+             encode_operand_map(&uc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
     if (!ok) {
         *why = "cuTensorMapEncodeTiled failed or is unavailable";
         return cudaErrorInvalidValue;
@@ -417,7 +416,7 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     if (tiles > uc.tiles_capacity) return cudaErrorInvalidValue;
     KernelParams p;
     p.alpha2 = uc.alpha2;
-    p.n_tile_blocks = (int)((tiles + uc.bn - 1) / uc.bn);
+    p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
     p.n_co_blocks = uc.n_co_blocks;
     p.bn = uc.bn;
     p.k_blocks = uc.k_blocks;

@@ -102,7 +102,7 @@ struct UmmaContract {
     int passes;        // 1 or 3
     int alpha2, Cout, cin_pad;
     long long tiles_capacity;
-    int bn;            // MMA N (tiles per work item), multiple of 16, <= 256
+    int bn;            // MMA N (output channels per work item), multiple of 16, <= 256
     int n_co_blocks;
     int k_blocks;
     int stages;
