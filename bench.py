@@ -27,6 +27,11 @@ if ROOT not in sys.path:
 METRIC = "conv TFLOP/s (direct-conv-equivalent)"
 UNIT = "TFLOP/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch (mean over the four layers of one step) from one ncu
+# capture of this file's default workload (profiles/bench_config1_b32_launch_list.md gives the command).  Valid
+# for config1_b32 / tf32 and the kernels as captured; set an entry to None when its kernel changes.
+NCU_DRAM_BYTES_PER_LAUNCH = {"config1_b32/tf32": {"input": 40.42e6, "contraction": 45.54e6, "output": 15.51e6}}
+
 
 def workload_layers(name: str):
     from paper_2002_12418_b200 import workloads as W
@@ -207,12 +212,15 @@ def stage_work(layer, info):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config1_b32")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--precision", default="tf32", choices=["tf32", "bf16"])
+    ap.add_argument("--calibration", default="measure", choices=["measure", "builtin"],
+                    help="measure: run mnn_calibrate on this GPU before planning (default); builtin: plan from the "
+                         "library's frozen B200 record (use under a profiler, which slows the calibration launches)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -244,8 +252,11 @@ def main():
     layers = workload_layers(args.workload)
     prec = B.PREC_TF32 if args.precision == "tf32" else B.PREC_BF16
     # pre-inference: the planner's cost constants are measured once on this GPU, before any plan is made
-    calibration = B.mnn_calibrate(local_rank, torch.cuda.current_stream(dev).cuda_stream)
-    torch.cuda.synchronize(dev)
+    if args.calibration == "measure":
+        calibration = B.mnn_calibrate(local_rank, torch.cuda.current_stream(dev).cuda_stream)
+        torch.cuda.synchronize(dev)
+    else:
+        calibration = B.mnn_get_calibration()
     # every rank works on its own batch of the same shape (weak scaling; images are independent)
     state = []
     for i, layer in enumerate(layers):
@@ -335,7 +346,9 @@ def main():
     dom_bytes = stage_bytes[dominant] / dom_launches
     achieved_gbs = dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
     roofline = {"kernel": dominant, "bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved_gbs / peaks["hbm_gbs"],
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get("%s/%s" % (args.workload, args.precision), {}).get(dominant),
+                "algorithmic_bytes_per_launch": dom_bytes, "peak_source": peaks["source"],
                 "avg_launch_us": dom_ms * 1e3, "launches": stage_n[dominant],
                 "stage_ms_per_step": {n: stage_ms[n] / args.steps for n in stage_names},
                 "stage_gbs": {n: (stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 if stage_ms[n] > 0 else None)
@@ -386,7 +399,7 @@ def main():
                 "data": "synthetic",
                 "config": {"workload": args.workload, "layers": len(layers), "batch_per_gpu": layers[0].N,
                            "l2": "flushed before every step (256 MB write)", "weights": "pre-transformed",
-                           "accuracy_class": args.precision, "planner_calibration": calibration[:9], "plans": per_layer},
+                           "accuracy_class": args.precision, "planner_calibration": calibration[:9], "calibration_source": args.calibration, "plans": per_layer},
                 "clocks": clocks, "roofline": roofline,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms / e2e_steps},
