@@ -354,11 +354,34 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
         *why = "operand rows must be a multiple of 16 bytes";
         return cudaErrorInvalidValue;
     }
-    // output channels per work item (MMA N): as many as fit (<= 256), multiple of 16, blocks balanced
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&uc->num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    // Output channels per work item (MMA N): a multiple of 16, at most 256, channel blocks balanced.  Wider
+    // blocks re-use the V tile more; narrower ones give more work items.  Among 1x, 2x and 4x the minimum
+    // number of blocks take the one with the shortest schedule: rounds of work items over the SMs times the
+    // operand rows an item loads (128 tiles + bn channels).
     {
         const int co16 = (Cout + 15) / 16 * 16;
-        uc->n_co_blocks = (co16 + 255) / 256;
-        uc->bn = ((co16 / 16 + uc->n_co_blocks - 1) / uc->n_co_blocks) * 16;
+        const int min_blocks = (co16 + 255) / 256;
+        const long long tile_blocks = (tiles_capacity + kTileM - 1) / kTileM;
+        long long best_cost = -1;
+        for (int mult = 1; mult <= 4; mult *= 2) {
+            const int blocks = min_blocks * mult;
+            const int bn = ((co16 / 16 + blocks - 1) / blocks) * 16;
+            if (bn < 32 && mult > 1) break;
+            const int real_blocks = (co16 + bn - 1) / bn;
+            const long long items = tile_blocks * real_blocks * alpha2;
+            const long long rounds = (items + uc->num_sms - 1) / uc->num_sms;
+            const long long cost = rounds * (kTileM + bn);
+            if (best_cost < 0 || cost < best_cost) {
+                best_cost = cost;
+                uc->bn = bn;
+                uc->n_co_blocks = real_blocks;
+            }
+        }
     }
     const int k_elems = kSwizzleBytes / eb;
     uc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
@@ -377,12 +400,6 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     int cols = 32;
     while (cols < 2 * uc->bn) cols *= 2;
     uc->tmem_cols = cols;
-
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&uc->num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
 
     const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
     bool ok = encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&

@@ -420,38 +420,49 @@ inline bool bt_has_symmetric_structure(const float* Bt, int alpha)
     return true;
 }
 
-// Item geometry: the longest segment for which at least three buffers fit shared memory.
-inline bool plan_input_items(const WinoGeom& g, int alpha, bool tma_ok, InputItems* it)
+// Item geometry.
+inline bool plan_input_items(const WinoGeom& g, int alpha, bool tma_ok, int num_sms, InputItems* it)
 {
     it->use_tma = tma_ok ? 1 : 0;
     it->vec = tma_ok ? 4 : ((g.W % 2 == 0) ? 2 : 1);
     it->loader_warps = tma_ok ? 1 : 8;
     it->cblocks = (g.cin_pad + kItChannels - 1) / kItChannels;
-    for (int nseg = 1; nseg <= g.tw; ++nseg) {
+    // Candidates: the longest segment for which at least three buffers fit, and up to three finer splits;
+    // the one with the shortest schedule wins (rounds of items over the SMs times tiles per item plus one
+    // tile's worth of per-item overhead).
+    long long best_cost = -1;
+    int found = 0;
+    for (int nseg = 1; nseg <= g.tw && found < 4; ++nseg) {
         const int txs = (g.tw + nseg - 1) / nseg;
+        if (nseg > 1 && txs == (g.tw + nseg - 2) / (nseg - 1)) continue;      // same segment length as before
         const int span = (txs - 1) * g.m + alpha;
         // staged columns: the span, what the vector grid adds in front (up to vec - 1) and what the compute
         // side may read beyond the last tile (whole 4-wide vectors), rounded up to 4 x odd
         int wb = (span + (it->vec - 1) + 3 + 3) / 4 * 4;
         if (((wb / 4) & 1) == 0) wb += 4;
         if (wb > 256) continue;
-        if (!tma_ok && alpha * (wb / it->vec) > 32 * kItCopySlots && txs > 1) continue;
+        if (!tma_ok && alpha * (wb / it->vec) > 32 * kItCopySlots) continue;
         const long long bytes = (long long)alpha * kItChannels * wb * 4;
         long long nbuf = kItSmemBudget / bytes;
-        if (nbuf >= 3 || txs == 1) {
-            if (nbuf < 2) return false;
-            if (!tma_ok && alpha * (wb / it->vec) > 32 * kItCopySlots) return false;
-            if (nbuf > kItMaxBuffers) nbuf = kItMaxBuffers;
+        if (nbuf < 3 && !(txs == 1 && nbuf >= 2)) continue;
+        if (nbuf > kItMaxBuffers) nbuf = kItMaxBuffers;
+        const int real_nseg = (g.tw + txs - 1) / txs;
+        const long long n_items = (long long)g.images * g.th * real_nseg * it->cblocks;
+        if (n_items >= (1ll << 31)) continue;
+        const long long rounds = (n_items + num_sms - 1) / num_sms;
+        const long long cost = rounds * (txs + 1);
+        ++found;
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
             it->txs = txs;
-            it->nseg = (g.tw + txs - 1) / txs;
+            it->nseg = real_nseg;
             it->wb = wb;
             it->nbuf = (int)nbuf;
             it->buf_words = alpha * kItChannels * wb;
-            it->n_items = (long long)g.images * g.th * it->nseg * it->cblocks;
-            return it->n_items < (1ll << 31);
+            it->n_items = n_items;
         }
     }
-    return false;
+    return best_cost >= 0;
 }
 
 // Defined beside the other tensor-map code (contract_umma.cu).
@@ -470,10 +481,10 @@ cudaError_t launch_input_ws(const float* x, void* V_hi, void* V_lo, const WinoGe
     CUtensorMap xmap;
     std::memset(&xmap, 0, sizeof(xmap));
     if (tma_ok) {
-        if (!plan_input_items(g, ALPHA, true, &it) || !encode_input_map(&xmap, x, g.images, g.Cin, g.H, g.W, it.wb, kPair))
+        if (!plan_input_items(g, ALPHA, true, num_sms, &it) || !encode_input_map(&xmap, x, g.images, g.Cin, g.H, g.W, it.wb, kPair))
             tma_ok = false;
     }
-    if (!tma_ok && !plan_input_items(g, ALPHA, false, &it)) return cudaErrorInvalidConfiguration;
+    if (!tma_ok && !plan_input_items(g, ALPHA, false, num_sms, &it)) return cudaErrorInvalidConfiguration;
     const size_t smem = (size_t)it.nbuf * it.buf_words * sizeof(float);
     long long grid = it.n_items < num_sms ? it.n_items : num_sms;
     if (grid <= 0) return cudaSuccess;
