@@ -212,7 +212,7 @@ def stage_work(layer, info):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config1_b32")
@@ -229,6 +229,7 @@ def main():
     import numpy as np
     import torch
     from paper_2002_12418_b200 import binding as B
+    from paper_2002_12418_b200 import replicas as R
     from paper_2002_12418_b200 import workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
@@ -260,7 +261,7 @@ def main():
     # every rank works on its own batch of the same shape (weak scaling; images are independent)
     state = []
     for i, layer in enumerate(layers):
-        lay = layer if world == 1 else layer.with_batch(layer.N, seed_offset=10000 * rank)
+        lay = layer if world == 1 else layer.with_batch(layer.N, seed_offset=R.rank_seed_offset(rank))
         x, w, b = W.make_inputs(lay)
         o = B.make_opts(groups=lay.groups, relu=lay.relu, precision=prec)
         r = B.ConvLayerRunner(lay.N, lay.Cin, lay.Cout, lay.H, lay.W, lay.k, lay.stride, lay.pad, lay.dilation, o,
@@ -302,12 +303,9 @@ def main():
     step_ms = [a.elapsed_time(b) for a, b in ev]
     clocks = sampler.stop(t_wall0, t_wall1)
     total_ms = float(sum(step_ms))
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = R.max_over_ranks(dist, total_ms, dev)
     flops_step = sum(s["layer"].direct_flops for s in state)
-    value = world * flops_step * args.steps / (total_ms * 1e-3) / 1e12
+    value = R.whole_job_throughput(flops_step, args.steps, world, total_ms)
     launches = sum(s["runner"].info.launches_per_run for s in state) * args.steps
 
     # ---- per-kernel durations (events around every launch), same steps again ----
@@ -379,11 +377,8 @@ def main():
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * flops_step * e2e_steps / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = R.max_over_ranks(dist, e2e_ms, dev)
+    e2e_value = R.whole_job_throughput(flops_step, e2e_steps, world, e2e_ms)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
