@@ -86,6 +86,67 @@ __global__ void __launch_bounds__(256) gather_kernel(const float* __restrict__ x
     }
 }
 
+// 1 x 1, stride 1, no padding: the gather is a transposition of each image from [channel][pixel] to
+// [pixel][channel] with rounding.  A CTA moves a 64 x 64 block through shared memory: 128-bit loads along
+// the pixels, 128-bit (fp32 containers) or 64-bit (bf16) stores along the channels.  Needs H * W % 4 == 0.
+template <int MODE>
+__global__ void __launch_bounds__(256) gather_1x1_kernel(const float* __restrict__ x, void* V_hi, void* V_lo, int Cin, int hw,
+                                                         int k_pad)
+{
+    __shared__ float tile[64][65];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int p0 = blockIdx.x * 64, c0 = blockIdx.y * 64, n = blockIdx.z;
+    const float* xn = x + (size_t)n * Cin * hw;
+    {
+        const int pv = (threadIdx.x & 15) * 4, cr = threadIdx.x >> 4;      // 16 vectors of 4 pixels x 16 channels
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = cr + 16 * i;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c0 + c < Cin && p0 + pv < hw) v = __ldg(reinterpret_cast<const float4*>(xn + (size_t)(c0 + c) * hw + p0 + pv));
+            tile[c][pv] = v.x; tile[c][pv + 1] = v.y; tile[c][pv + 2] = v.z; tile[c][pv + 3] = v.w;
+        }
+    }
+    __syncthreads();
+    const int cv = (threadIdx.x & 15) * 4, pr = threadIdx.x >> 4;          // 16 vectors of 4 channels x 16 pixels
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int p = pr + 16 * i;
+        if (p0 + p >= hw || c0 + cv >= k_pad) continue;
+        const size_t idx = ((size_t)n * hw + p0 + p) * k_pad + c0 + cv;     // multiple of 4: k_pad is a multiple of 8
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = tile[cv + e][p];
+        if (MODE == STORE_BF16 || MODE == STORE_BF16_SPLIT) {
+            __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&h01);
+            pk.y = *reinterpret_cast<uint32_t*>(&h23);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(V_hi) + idx) = pk;
+            if (MODE == STORE_BF16_SPLIT) {
+                const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+                __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y),
+                               l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+                pk.x = *reinterpret_cast<uint32_t*>(&l01);
+                pk.y = *reinterpret_cast<uint32_t*>(&l23);
+                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(V_lo) + idx) = pk;
+            }
+        } else if (MODE == STORE_FP32) {
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_hi) + idx) = make_float4(v[0], v[1], v[2], v[3]);
+        } else {
+            float h[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) h[e] = round_tf32_g(v[e]);
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_hi) + idx) = make_float4(h[0], h[1], h[2], h[3]);
+            if (MODE == STORE_TF32_SPLIT)
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_lo) + idx) =
+                    make_float4(round_tf32_g(v[0] - h[0]), round_tf32_g(v[1] - h[1]), round_tf32_g(v[2] - h[2]),
+                                round_tf32_g(v[3] - h[3]));
+        }
+    }
+}
+
 // Generic direct convolution: one thread per output element.
 __global__ void __launch_bounds__(256) direct_generic_kernel(const float* __restrict__ x, const float* __restrict__ w,
                                                              const float* __restrict__ bias, float* __restrict__ y,
@@ -226,6 +287,17 @@ cudaError_t launch_gather(const float* x, void* V_hi, void* V_lo, const GatherGe
 {
     const long long T = (long long)g.N * g.OH * g.OW;
     if (T <= 0) return cudaSuccess;
+    const int hw = g.H * g.W;
+    if (g.k == 1 && g.stride == 1 && g.pad == 0 && hw % 4 == 0 && g.N <= 65535 && (g.k_pad + 63) / 64 <= 65535) {
+        const dim3 grid((unsigned)((hw + 63) / 64), (unsigned)((g.k_pad + 63) / 64), (unsigned)g.N);
+        switch (mode) {
+            case STORE_TF32: return launch_overlapped(gather_1x1_kernel<STORE_TF32>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
+            case STORE_BF16: return launch_overlapped(gather_1x1_kernel<STORE_BF16>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
+            case STORE_TF32_SPLIT: return launch_overlapped(gather_1x1_kernel<STORE_TF32_SPLIT>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
+            case STORE_BF16_SPLIT: return launch_overlapped(gather_1x1_kernel<STORE_BF16_SPLIT>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
+            default: return launch_overlapped(gather_1x1_kernel<STORE_FP32>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
+        }
+    }
     const long long bx = (T + 31) / 32;
     const int by = (g.k_pad + 31) / 32;
     if (bx > 2147483647ll || by > 65535) return cudaErrorInvalidValue;
