@@ -26,7 +26,7 @@ namespace {
 constexpr int kThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int kTileM = 128;            // tiles (rows of V) per work item
 constexpr int kMaxStages = 8;
-constexpr int kMaxSharedBias = 2048;    // output channels whose bias is staged in shared memory
+constexpr int kMaxSharedBias = 2048;    // output channels whose bias is staged in shared memory (+ 16 of slack)
 constexpr int kSwizzleBytes = 128;     // bytes of K per shared-memory row
 constexpr int kSmemBudget = 200 * 1024;
 
@@ -55,7 +55,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     __shared__ __align__(8) uint64_t tempty_bar[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ __align__(16) float s_bias[kMaxSharedBias];   // GEMM scheme: bias (zeros if none) for the epilogue
+    __shared__ __align__(16) float s_bias[kMaxSharedBias + 16];   // GEMM scheme: bias (zeros if none) for the epilogue
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -222,23 +222,49 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 ptx::tmem_ld_wait();
                 if (t_ok) {
                     const int n = min(16, n_co - c0);
+                    float* pj = dst;                                   // walks the 16 channels of this chunk
                     if (p.epi.mode == 0) {
                         if (n == 16) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) dst[(long long)j * step] = __uint_as_float(v[j]);
+                            for (int j = 0; j < 16; ++j) {
+                                *pj = __uint_as_float(v[j]);
+                                pj += step;
+                            }
                         } else {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (j < n) dst[(long long)j * step] = __uint_as_float(v[j]);
+                            for (int j = 0; j < 16; ++j) {
+                                if (j < n) *pj = __uint_as_float(v[j]);
+                                pj += step;
+                            }
                         }
                     } else {
+                        float bz[16];
+                        if (bias_in_smem) {
+                            // (reads past Cout stay inside the array and are not used)
+                            const float4* bp = reinterpret_cast<const float4*>(s_bias + co0 + c0);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (j < n) {
-                                float o = __uint_as_float(v[j]) + (bias_in_smem ? s_bias[co0 + c0 + j]
-                                                                                : (p.epi.bias ? __ldg(p.epi.bias + co0 + c0 + j) : 0.0f));
-                                if (p.epi.relu) o = fmaxf(o, 0.0f);
-                                dst[(long long)j * step] = o;
+                            for (int j = 0; j < 4; ++j) {
+                                const float4 q4 = bp[j];
+                                bz[4 * j] = q4.x; bz[4 * j + 1] = q4.y; bz[4 * j + 2] = q4.z; bz[4 * j + 3] = q4.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) bz[j] = (p.epi.bias && j < n) ? __ldg(p.epi.bias + co0 + c0 + j) : 0.0f;
+                        }
+                        const bool relu = p.epi.relu != 0;
+                        if (n == 16) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float o = __uint_as_float(v[j]) + bz[j];
+                                *pj = relu ? fmaxf(o, 0.0f) : o;
+                                pj += step;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float o = __uint_as_float(v[j]) + bz[j];
+                                if (j < n) *pj = relu ? fmaxf(o, 0.0f) : o;
+                                pj += step;
                             }
                         }
                     }
