@@ -362,18 +362,43 @@ def main():
         s["y_pin"] = torch.empty(s["y"].shape, dtype=torch.float32).pin_memory()
     e2e_steps = max(3, min(args.steps, 10))
 
+    # Three streams, linked by events: the copy of layer i + 1's input and the read-back of layer i - 1's
+    # result run while layer i computes (the GPU's copy engines work in both directions at once).
+    h2d_stream, d2h_stream = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    for s in state:
+        s["x_ready"], s["x_free"] = torch.cuda.Event(), torch.cuda.Event()
+        s["y_ready"], s["y_free"] = torch.cuda.Event(), torch.cuda.Event()
+        s["x_free"].record(stream)
+        s["y_free"].record(stream)
+
     def e2e_step():
         for s in state:
-            s["x"].copy_(s["x_pin"], non_blocking=True)
+            with torch.cuda.stream(h2d_stream):
+                h2d_stream.wait_event(s["x_free"])               # the previous pass over this layer has read x
+                s["x"].copy_(s["x_pin"], non_blocking=True)
+                s["x_ready"].record(h2d_stream)
+            stream.wait_event(s["x_ready"])
+            stream.wait_event(s["y_free"])                       # the previous result has been read back
             s["runner"].run(s["x"], s["w"], s["b"], s["y"])
-            s["y_pin"].copy_(s["y"], non_blocking=True)
+            s["x_free"].record(stream)
+            s["y_ready"].record(stream)
+            with torch.cuda.stream(d2h_stream):
+                d2h_stream.wait_event(s["y_ready"])
+                s["y_pin"].copy_(s["y"], non_blocking=True)
+                s["y_free"].record(d2h_stream)
+
+    def e2e_join():
+        for s in state:
+            stream.wait_event(s["y_free"])
 
     e2e_step()
+    e2e_join()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
+    e2e_join()
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
