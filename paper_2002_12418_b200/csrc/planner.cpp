@@ -37,12 +37,12 @@ Calibration default_calibration()
     Calibration c;
     std::memset(&c, 0, sizeof(c));
     // one calibration record measured on a B200 (mnn_calibrate), rounded
-    c.c[0] = 171000;      // as per HBM byte          (~5.8 TB/s with a plain copy kernel)
-    c.c[1] = 75000;       // as per L2-resident byte  (~13 TB/s)
-    c.c[2] = 2440;        // as per TF32 tensor flop  (~410 TFLOP/s achieved by the contraction kernel)
-    c.c[3] = 1390;        // as per BF16 tensor flop  (~720 TFLOP/s achieved)
+    c.c[0] = 173000;      // as per HBM byte          (~5.8 TB/s with a plain copy kernel)
+    c.c[1] = 84000;       // as per L2-resident byte  (~12 TB/s)
+    c.c[2] = 1930;        // as per TF32 tensor flop  (~520 TFLOP/s achieved by the contraction kernel)
+    c.c[3] = 1050;        // as per BF16 tensor flop  (~950 TFLOP/s achieved)
     c.c[4] = 28000;       // as per fp32 ALU flop in the transform kernels (~36 TFLOP/s)
-    c.c[5] = 5500000;     // ps of fixed cost per kernel: launch, ramp-up and tail (the t_schedule of Eq. 5)
+    c.c[5] = 3530000;     // ps of fixed cost per kernel: launch, ramp-up and tail (the t_schedule of Eq. 5)
     c.c[6] = 80ll << 20;  // L2 bytes one chunk's V + M may occupy
     c.c[7] = 148;         // SMs
     c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
@@ -326,8 +326,9 @@ uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes
     const uint64_t y_bytes = 4ull * n * s.Cout * s.OH * s.OW;
     const uint64_t cV = (uint64_t)(resident ? cal.c[1] : cal.c[0]);
     const uint64_t c0 = (uint64_t)cal.c[0], cA = (uint64_t)cal.c[4];
-    // from alpha = 8 on a lane of the input transform holds one channel instead of a packed pair: twice the ALU time
-    const uint64_t in_alu = (alpha >= 8 ? 2ull : 1ull) * 4ull * alpha * a2 * n * tiles_img * s.Cin * cA;
+    // from alpha = 8 on a lane of the input transform holds one channel instead of a packed pair (twice the ALU
+    // time); from alpha = 10 on the tile no longer fits the register file (measured about twice that again)
+    const uint64_t in_alu = (alpha >= 10 ? 4ull : (alpha >= 8 ? 2ull : 1ull)) * 4ull * alpha * a2 * n * tiles_img * s.Cin * cA;
     const uint64_t in = kernel_ps(x_bytes * c0 + v_bytes * cV, 0, in_alu, cal);
     const uint64_t con = kernel_ps((v_bytes + m_bytes) * cV + u_bytes * c0,
                                    2ull * a2 * s.Cout * Cp * n * tiles_img * passes * tensor_as(operand, cal), 0, cal);
