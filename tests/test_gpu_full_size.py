@@ -144,3 +144,33 @@ def test_networks_large_batch_sampled(torch, which):
             assert info.algo == B.ALGO_GEMM, layer.name          # ... and 1x1 layers through the matrix product
         if layer.groups > 1:
             assert info.algo == B.ALGO_DIRECT, layer.name
+
+
+@pytest.mark.parametrize("m,k,H,C,N,operand,passes", [
+    (2, 3, 56, 128, 16, B.OPERAND_TF32, 1),      # alpha 4, TMA rows, channel pairs
+    (4, 3, 56, 128, 16, B.OPERAND_BF16, 3),      # alpha 6
+    (6, 3, 56, 128, 16, B.OPERAND_BF16, 3),      # alpha 8, one channel per lane, 4-D row boxes
+    (2, 7, 28, 128, 32, B.OPERAND_TF32, 3),      # alpha 8 from a 7x7 kernel
+    (4, 3, 30, 96, 24, B.OPERAND_BF16, 3),       # rows not 16-byte aligned: cp.async loaders
+    (2, 3, 14, 256, 64, B.OPERAND_TF32, 1)])
+def test_many_work_items_per_cta_are_repeatable(torch, m, k, H, C, N, operand, passes):
+    """Several ring-buffer rounds per CTA in every kernel of the pipeline; ten runs must agree bit for bit
+    (a buffer handed over too early shows up as run-to-run differences) and match the oracle on samples."""
+    layer = W.ConvLayer("t", N, C, C, H, H, k, 1, k // 2, relu=True, seed=4242 + m + k)
+    inputs = W.make_inputs(layer)
+    x, w, b = inputs
+    o = B.make_opts(relu=1, force_algo=B.ALGO_WINOGRAD, force_m=m, operand=operand, passes=passes)
+    r = B.ConvLayerRunner(N, C, C, H, H, k, 1, k // 2, 1, o)
+    xd, wd, bd = to_dev(torch, x), to_dev(torch, w), to_dev(torch, b)
+    first = None
+    for i in range(10):
+        y = r.run(xd, wd, bd)
+        torch.cuda.synchronize()
+        assert r.device_status() == 0
+        if first is None:
+            first = y.clone()
+        else:
+            assert torch.equal(y, first), "run %d differs from run 0" % i
+    got = first.cpu().numpy()
+    r.close()
+    check_sampled(layer, got, inputs, B.PREC_TF32)
