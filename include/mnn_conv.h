@@ -240,6 +240,57 @@ MNN_API int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CONST
 MNN_API int mnn_set_calibration(const long long consts[MNN_N_CONSTS]);
 MNN_API int mnn_get_calibration(long long consts[MNN_N_CONSTS]);
 
+/*
+ * Network-level pre-inference (Section 3.2, "preparation-execution decoupling": the
+ * engine walks the graph once, decides every scheme and lays out all memory before the
+ * first inference).  A network here is a sequential stack of convolution layers on one
+ * input of shape [N][layers[0].Cin][H][W]; layer i consumes layer i-1's output.
+ *
+ * mnn_net_plan plans every layer (same options as mnn_conv_plan_ex: accuracy class
+ * `precision`; groups / relu per layer) and lays out ONE workspace by a virtual walk:
+ *   - a persistent part per layer (status word and transformed weights U),
+ *   - one transient part shared by all layers (V and M of the largest layer),
+ *   - two activation buffers used in turn, each as large as the largest intermediate tensor.
+ * mnn_net_query reports the layout and each layer's plan; mnn_net_set_workspace hands over
+ * the caller-owned workspace (1024-byte aligned, >= info.workspace_bytes);
+ * mnn_net_prepare transforms all weights; mnn_net_run enqueues the whole forward pass
+ * on `stream` (x -> y; w[i], bias[i] are the layers' device tensors, bias[i] may be NULL)
+ * with no allocation, no synchronisation and no host work beyond the kernel launches, so
+ * that it can also be recorded once (e.g. into a CUDA graph) and replayed.
+ * Layers run in order on one stream: the shared transient part is safe by stream order.
+ */
+typedef struct mnn_net_s* mnn_net_t;
+
+typedef struct {
+    int Cin, Cout, k, stride, pad, dilation;
+    int groups;        /* 0 or 1, or Cin (= Cout) for depthwise */
+    int relu;
+} mnn_layer_desc;
+
+#define MNN_NET_MAX_LAYERS 128
+typedef struct {
+    int n_layers;
+    int N, H, W;                       /* input */
+    int out_C, out_H, out_W;           /* output of the last layer */
+    int launches_per_run;
+    long long workspace_bytes;         /* total the caller must provide */
+    long long persistent_bytes, transient_bytes, activation_bytes;   /* activation_bytes = one of the two buffers */
+    long long sum_of_layer_workspaces; /* what per-layer workspaces would need without sharing */
+    int algo[MNN_NET_MAX_LAYERS], m[MNN_NET_MAX_LAYERS], operand[MNN_NET_MAX_LAYERS], passes[MNN_NET_MAX_LAYERS];
+    int OH[MNN_NET_MAX_LAYERS], OW[MNN_NET_MAX_LAYERS];
+} mnn_net_info;
+
+MNN_API mnn_net_t mnn_net_plan(int N, int H, int W, int n_layers, const mnn_layer_desc* layers, int precision);
+MNN_API int mnn_net_query(mnn_net_t net, mnn_net_info* info);
+MNN_API int mnn_net_set_workspace(mnn_net_t net, void* workspace, long long bytes);
+MNN_API int mnn_net_prepare(mnn_net_t net, const float* const* w, void* stream);
+MNN_API int mnn_net_run(mnn_net_t net, const float* x, const float* const* w, const float* const* bias, float* y,
+                        void* stream);
+/* Reads and clears the status words of all layers (synchronises the stream); *code gets the first
+ * non-zero code, *layer its index (-1 if none). */
+MNN_API int mnn_net_device_status(mnn_net_t net, void* stream, int* code, int* layer);
+MNN_API void mnn_net_destroy(mnn_net_t net);
+
 MNN_API const char* mnn_last_error(void);
 
 #ifdef __cplusplus

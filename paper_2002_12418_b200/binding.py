@@ -26,7 +26,10 @@ OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "
 EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_query", "mnn_conv_set_workspace",
             "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
             "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
-            "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error"]
+            "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error",
+            "mnn_net_plan", "mnn_net_query", "mnn_net_set_workspace", "mnn_net_prepare", "mnn_net_run",
+            "mnn_net_device_status", "mnn_net_destroy"]
+NET_MAX_LAYERS = 128
 
 
 class ConvOpts(ctypes.Structure):
@@ -49,6 +52,23 @@ class ConvInfo(ctypes.Structure):
                 ("predicted_error_ppm", ctypes.c_longlong),
                 ("chosen_candidate", ctypes.c_int), ("reserved", ctypes.c_int),
                 ("cost_ps", ctypes.c_ulonglong * N_CANDIDATES)]
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [("Cin", ctypes.c_int), ("Cout", ctypes.c_int), ("k", ctypes.c_int), ("stride", ctypes.c_int),
+                ("pad", ctypes.c_int), ("dilation", ctypes.c_int), ("groups", ctypes.c_int), ("relu", ctypes.c_int)]
+
+
+class NetInfo(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int), ("N", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int),
+                ("out_C", ctypes.c_int), ("out_H", ctypes.c_int), ("out_W", ctypes.c_int),
+                ("launches_per_run", ctypes.c_int),
+                ("workspace_bytes", ctypes.c_longlong), ("persistent_bytes", ctypes.c_longlong),
+                ("transient_bytes", ctypes.c_longlong), ("activation_bytes", ctypes.c_longlong),
+                ("sum_of_layer_workspaces", ctypes.c_longlong),
+                ("algo", ctypes.c_int * NET_MAX_LAYERS), ("m", ctypes.c_int * NET_MAX_LAYERS),
+                ("operand", ctypes.c_int * NET_MAX_LAYERS), ("passes", ctypes.c_int * NET_MAX_LAYERS),
+                ("OH", ctypes.c_int * NET_MAX_LAYERS), ("OW", ctypes.c_int * NET_MAX_LAYERS)]
 
 
 class MnnError(RuntimeError):
@@ -102,6 +122,20 @@ def lib():
         L.mnn_set_calibration.restype = i
         L.mnn_get_calibration.argtypes = [ctypes.POINTER(ll)]
         L.mnn_get_calibration.restype = i
+        L.mnn_net_plan.argtypes = [i, i, i, i, ctypes.POINTER(LayerDesc), i]
+        L.mnn_net_plan.restype = p
+        L.mnn_net_query.argtypes = [p, ctypes.POINTER(NetInfo)]
+        L.mnn_net_query.restype = i
+        L.mnn_net_set_workspace.argtypes = [p, p, ll]
+        L.mnn_net_set_workspace.restype = i
+        L.mnn_net_prepare.argtypes = [p, ctypes.POINTER(p), p]
+        L.mnn_net_prepare.restype = i
+        L.mnn_net_run.argtypes = [p, p, ctypes.POINTER(p), ctypes.POINTER(p), p, p]
+        L.mnn_net_run.restype = i
+        L.mnn_net_device_status.argtypes = [p, p, ctypes.POINTER(i), ctypes.POINTER(i)]
+        L.mnn_net_device_status.restype = i
+        L.mnn_net_destroy.argtypes = [p]
+        L.mnn_net_destroy.restype = None
         L.mnn_last_error.argtypes = []
         L.mnn_last_error.restype = ctypes.c_char_p
         _lib = L
@@ -225,6 +259,98 @@ def mnn_get_calibration() -> list[int]:
     c = (ctypes.c_longlong * N_CONSTS)()
     _check(lib().mnn_get_calibration(c))
     return list(c)
+
+
+def mnn_net_plan(N, H, W, layers, precision=PREC_TF32):
+    """layers: sequence of objects with Cin, Cout, k, stride, pad, dilation, groups, relu (e.g. workloads.ConvLayer)."""
+    arr = (LayerDesc * len(layers))()
+    for d, l in zip(arr, layers):
+        d.Cin, d.Cout, d.k, d.stride, d.pad, d.dilation = l.Cin, l.Cout, l.k, l.stride, l.pad, l.dilation
+        d.groups, d.relu = l.groups, int(bool(l.relu))
+    h = lib().mnn_net_plan(N, H, W, len(layers), arr, precision)
+    if not h:
+        raise MnnError(MNN_EINVAL, mnn_last_error())
+    return h
+
+
+def mnn_net_query(net) -> NetInfo:
+    info = NetInfo()
+    _check(lib().mnn_net_query(net, ctypes.byref(info)))
+    return info
+
+
+def _ptr_array(ptrs):
+    return (ctypes.c_void_p * len(ptrs))(*[ctypes.c_void_p(v) if v else None for v in ptrs])
+
+
+def mnn_net_set_workspace(net, ptr: int, nbytes: int) -> None:
+    _check(lib().mnn_net_set_workspace(net, ptr, nbytes))
+
+
+def mnn_net_prepare(net, w_ptrs, stream: int) -> None:
+    _check(lib().mnn_net_prepare(net, _ptr_array(w_ptrs), stream))
+
+
+def mnn_net_run(net, x_ptr: int, w_ptrs, bias_ptrs, y_ptr: int, stream: int) -> None:
+    _check(lib().mnn_net_run(net, x_ptr, _ptr_array(w_ptrs), _ptr_array(bias_ptrs), y_ptr, stream))
+
+
+def mnn_net_device_status(net, stream: int):
+    code, layer = ctypes.c_int(0), ctypes.c_int(-1)
+    _check(lib().mnn_net_device_status(net, stream, ctypes.byref(code), ctypes.byref(layer)))
+    return code.value, layer.value
+
+
+def mnn_net_destroy(net) -> None:
+    lib().mnn_net_destroy(net)
+
+
+class NetRunner:
+    """A network plan plus its torch-owned workspace; ``run`` is one mnn_net_run on torch's current stream."""
+
+    def __init__(self, N, H, W, layers, precision=PREC_TF32, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.device = torch.device(device)
+        self.net = mnn_net_plan(N, H, W, layers, precision)
+        self.info = mnn_net_query(self.net)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(self.info.workspace_bytes + 1024, dtype=torch.uint8, device=self.device)
+        self._ws_ptr = (self.workspace.data_ptr() + 1023) // 1024 * 1024
+        mnn_net_set_workspace(self.net, self._ws_ptr, self.info.workspace_bytes)
+        self._keep = None
+
+    def stream(self) -> int:
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def prepare(self, ws) -> None:
+        mnn_net_prepare(self.net, [w.data_ptr() for w in ws], self.stream())
+
+    def bind(self, ws, bs) -> None:
+        """Marshal the weight / bias pointer arrays once (they are reused by every run)."""
+        self._keep = (_ptr_array([w.data_ptr() for w in ws]), _ptr_array([b.data_ptr() if b is not None else 0 for b in bs]))
+
+    def run(self, x, y=None):
+        torch = self.torch
+        if y is None:
+            y = torch.empty((self.info.N, self.info.out_C, self.info.out_H, self.info.out_W), dtype=torch.float32,
+                            device=self.device)
+        _check(lib().mnn_net_run(self.net, x.data_ptr(), self._keep[0], self._keep[1], y.data_ptr(), self.stream()))
+        return y
+
+    def device_status(self):
+        return mnn_net_device_status(self.net, self.stream())
+
+    def close(self) -> None:
+        if self.net:
+            mnn_net_destroy(self.net)
+            self.net = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class ConvLayerRunner:

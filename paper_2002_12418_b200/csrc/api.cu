@@ -49,7 +49,8 @@ struct mnn_conv_plan_s {
     int launches_per_run = 1;
     TransformMatrices mats;
     // run-time state
-    char* ws = nullptr;
+    char* ws = nullptr;              // status word and U (persistent part), and V, M unless tws is set
+    char* tws = nullptr;             // optional separate transient part: V at tws, M at tws + (m_offset - v_offset)
     long long ws_bytes = 0;
     const float* prepared_w = nullptr;
     UmmaContract uc;
@@ -63,9 +64,13 @@ namespace {
 
 void* u_hi(mnn_conv_plan_t p) { return p->ws + p->u_offset; }
 void* u_lo(mnn_conv_plan_t p) { return store_is_split(p->store_mode) ? p->ws + p->u_offset + p->u_bytes / 2 : nullptr; }
-void* v_hi(mnn_conv_plan_t p) { return p->ws + p->v_offset; }
-void* v_lo(mnn_conv_plan_t p) { return store_is_split(p->store_mode) ? p->ws + p->v_offset + p->v_bytes / 2 : nullptr; }
-float* m_buf(mnn_conv_plan_t p) { return reinterpret_cast<float*>(p->ws + p->m_offset); }
+char* transient_base(mnn_conv_plan_t p) { return p->tws ? p->tws - p->v_offset : p->ws; }
+void* v_hi(mnn_conv_plan_t p) { return transient_base(p) + p->v_offset; }
+void* v_lo(mnn_conv_plan_t p)
+{
+    return store_is_split(p->store_mode) ? transient_base(p) + p->v_offset + p->v_bytes / 2 : nullptr;
+}
+float* m_buf(mnn_conv_plan_t p) { return reinterpret_cast<float*>(transient_base(p) + p->m_offset); }
 int* status_word(mnn_conv_plan_t p) { return reinterpret_cast<int*>(p->ws); }
 
 int store_mode_of(int operand, int passes)
@@ -270,18 +275,52 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     return MNN_OK;
 }
 
+// Workspace in two parts (used by the network plan): `persistent` holds the status word and U
+// (the first v_offset bytes of the single-workspace layout), `transient` holds V and M and may be shared
+// with other plans that run on the same stream.
+static int set_workspace_split(mnn_conv_plan_t p, void* persistent, long long persistent_bytes, void* transient,
+                               long long transient_bytes);
+
 int mnn_conv_set_workspace(mnn_conv_plan_t p, void* workspace, long long bytes)
 {
     if (!p) return fail(MNN_EINVAL, "NULL plan");
+    if (p->workspace_bytes == 0) {
+        p->prepared_w = nullptr;
+        p->uc.ready = false;
+        p->ws = p->tws = nullptr;
+        p->ws_bytes = 0;
+        return MNN_OK;
+    }
+    if (!workspace) {
+        p->ws = p->tws = nullptr;
+        return fail(MNN_EWORKSPACE, "this plan needs a workspace");
+    }
+    if (bytes < p->workspace_bytes) {
+        p->ws = p->tws = nullptr;
+        return fail(MNN_EWORKSPACE, "workspace smaller than info.workspace_bytes");
+    }
+    return set_workspace_split(p, workspace, bytes, nullptr, 0);
+}
+
+static int set_workspace_split(mnn_conv_plan_t p, void* persistent, long long persistent_bytes, void* transient,
+                               long long transient_bytes)
+{
     p->prepared_w = nullptr;
     p->uc.ready = false;
-    p->ws = nullptr;
+    p->ws = p->tws = nullptr;
     p->ws_bytes = 0;
     if (p->workspace_bytes == 0) return MNN_OK;
-    if (!workspace) return fail(MNN_EWORKSPACE, "this plan needs a workspace");
-    if (bytes < p->workspace_bytes) return fail(MNN_EWORKSPACE, "workspace smaller than info.workspace_bytes");
+    void* workspace = persistent;
+    long long bytes = persistent_bytes;
+    if (!persistent) return fail(MNN_EWORKSPACE, "this plan needs a workspace");
+    if (transient) {
+        if (persistent_bytes < p->v_offset || transient_bytes < p->workspace_bytes - p->v_offset)
+            return fail(MNN_EWORKSPACE, "workspace part too small");
+        if (reinterpret_cast<uintptr_t>(transient) & 1023u) return fail(MNN_EALIGN, "workspace must be 1024-byte aligned");
+    }
     if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return fail(MNN_EALIGN, "workspace must be 1024-byte aligned");
     p->ws = static_cast<char*>(workspace);
+    p->tws = static_cast<char*>(transient);
     p->ws_bytes = bytes;
     cudaError_t e = cudaMemset(p->ws, 0, kStatusBytes);
     if (e != cudaSuccess) return fail_cuda(e, "clearing the status word");
@@ -538,6 +577,173 @@ int mnn_get_calibration(long long consts[MNN_N_CONSTS])
 }  // extern "C"
 
 // ---------------------------------------------------------------------------
+// Network-level plan: a sequential stack of layers, one workspace laid out by a virtual walk.
+// ---------------------------------------------------------------------------
+struct mnn_net_s {
+    int N = 0, H = 0, W = 0;
+    std::vector<mnn_conv_plan_t> plans;
+    std::vector<long long> persistent_offset;      // per layer, from the workspace base
+    long long persistent_bytes = 0, transient_bytes = 0, activation_bytes = 0, workspace_bytes = 0;
+    long long sum_of_layer_workspaces = 0;
+    long long transient_offset = 0, act_offset[2] = {0, 0};
+    char* ws = nullptr;
+    ~mnn_net_s()
+    {
+        for (mnn_conv_plan_t p : plans) mnn_conv_destroy(p);
+    }
+};
+
+extern "C" {
+
+mnn_net_t mnn_net_plan(int N, int H, int W, int n_layers, const mnn_layer_desc* layers, int precision)
+{
+    if (n_layers < 1 || n_layers > MNN_NET_MAX_LAYERS || !layers) {
+        fail(MNN_EINVAL, "a network needs 1..MNN_NET_MAX_LAYERS layers");
+        return nullptr;
+    }
+    mnn_net_t net = new (std::nothrow) mnn_net_s();
+    if (!net) {
+        fail(MNN_EINVAL, "out of host memory");
+        return nullptr;
+    }
+    net->N = N; net->H = H; net->W = W;
+    int c = layers[0].Cin, h = H, w = W;
+    long long off = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const mnn_layer_desc& L = layers[i];
+        if (L.Cin != c) {
+            fail(MNN_EINVAL, "layer " + std::to_string(i) + ": Cin does not match the previous layer's Cout");
+            delete net;
+            return nullptr;
+        }
+        mnn_conv_opts o;
+        std::memset(&o, 0, sizeof(o));
+        o.groups = L.groups ? L.groups : 1;
+        o.relu = L.relu;
+        o.precision = precision;
+        mnn_conv_plan_t p = mnn_conv_plan_ex(N, L.Cin, L.Cout, h, w, L.k, L.stride, L.pad, L.dilation, &o);
+        if (!p) {
+            g_last_error = "layer " + std::to_string(i) + ": " + g_last_error;
+            delete net;
+            return nullptr;
+        }
+        net->plans.push_back(p);
+        // virtual walk: the persistent part (status word + U) gets its own place, the transient part
+        // (V + M) only counts towards the maximum, the output towards the activation buffers
+        const long long persistent = p->workspace_bytes > 0 ? align_up(p->v_offset, 1024) : 0;
+        const long long transient = p->workspace_bytes > 0 ? p->workspace_bytes - p->v_offset : 0;
+        net->persistent_offset.push_back(off);
+        off += persistent;
+        if (transient > net->transient_bytes) net->transient_bytes = transient;
+        net->sum_of_layer_workspaces += p->workspace_bytes;
+        if (i + 1 < n_layers) {
+            const long long act = 4ll * N * L.Cout * p->s.OH * p->s.OW;
+            if (act > net->activation_bytes) net->activation_bytes = act;
+        }
+        c = L.Cout; h = p->s.OH; w = p->s.OW;
+    }
+    net->persistent_bytes = off;
+    net->transient_bytes = align_up(net->transient_bytes, 1024);
+    net->activation_bytes = align_up(net->activation_bytes, 1024);
+    net->transient_offset = net->persistent_bytes;
+    net->act_offset[0] = net->transient_offset + net->transient_bytes;
+    net->act_offset[1] = net->act_offset[0] + net->activation_bytes;
+    net->workspace_bytes = net->act_offset[1] + net->activation_bytes;
+    return net;
+}
+
+int mnn_net_query(mnn_net_t net, mnn_net_info* info)
+{
+    if (!net || !info) return fail(MNN_EINVAL, "NULL network or info");
+    std::memset(info, 0, sizeof(*info));
+    info->n_layers = (int)net->plans.size();
+    info->N = net->N; info->H = net->H; info->W = net->W;
+    info->workspace_bytes = net->workspace_bytes;
+    info->persistent_bytes = net->persistent_bytes;
+    info->transient_bytes = net->transient_bytes;
+    info->activation_bytes = net->activation_bytes;
+    info->sum_of_layer_workspaces = net->sum_of_layer_workspaces;
+    for (size_t i = 0; i < net->plans.size(); ++i) {
+        mnn_conv_plan_t p = net->plans[i];
+        info->algo[i] = p->d.algo; info->m[i] = p->d.m; info->operand[i] = p->d.operand; info->passes[i] = p->d.passes;
+        info->OH[i] = p->s.OH; info->OW[i] = p->s.OW;
+        info->launches_per_run += p->launches_per_run;
+    }
+    mnn_conv_plan_t last = net->plans.back();
+    info->out_C = last->s.Cout; info->out_H = last->s.OH; info->out_W = last->s.OW;
+    return MNN_OK;
+}
+
+int mnn_net_set_workspace(mnn_net_t net, void* workspace, long long bytes)
+{
+    if (!net) return fail(MNN_EINVAL, "NULL network");
+    net->ws = nullptr;
+    if (!workspace) return fail(MNN_EWORKSPACE, "the network needs a workspace");
+    if (bytes < net->workspace_bytes) return fail(MNN_EWORKSPACE, "workspace smaller than info.workspace_bytes");
+    if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return fail(MNN_EALIGN, "workspace must be 1024-byte aligned");
+    char* base = static_cast<char*>(workspace);
+    for (size_t i = 0; i < net->plans.size(); ++i) {
+        mnn_conv_plan_t p = net->plans[i];
+        if (p->workspace_bytes == 0) continue;
+        int rc = set_workspace_split(p, base + net->persistent_offset[i], align_up(p->v_offset, 1024),
+                                     base + net->transient_offset, net->transient_bytes);
+        if (rc != MNN_OK) return rc;
+    }
+    net->ws = base;
+    return MNN_OK;
+}
+
+int mnn_net_prepare(mnn_net_t net, const float* const* w, void* stream)
+{
+    if (!net || !w) return fail(MNN_EINVAL, "NULL network or weights");
+    if (!net->ws) return fail(MNN_EWORKSPACE, "call mnn_net_set_workspace first");
+    for (size_t i = 0; i < net->plans.size(); ++i) {
+        int rc = mnn_conv_prepare_weights(net->plans[i], w[i], stream);
+        if (rc != MNN_OK) return rc;
+    }
+    return MNN_OK;
+}
+
+int mnn_net_run(mnn_net_t net, const float* x, const float* const* w, const float* const* bias, float* y, void* stream)
+{
+    if (!net || !x || !w || !y) return fail(MNN_EINVAL, "NULL argument");
+    if (!net->ws) return fail(MNN_EWORKSPACE, "call mnn_net_set_workspace first");
+    const size_t n = net->plans.size();
+    const float* in = x;
+    for (size_t i = 0; i < n; ++i) {
+        float* out = i + 1 == n ? y : reinterpret_cast<float*>(net->ws + net->act_offset[i & 1]);
+        int rc = mnn_conv_run(net->plans[i], in, w[i], bias ? bias[i] : nullptr, out, stream);
+        if (rc != MNN_OK) {
+            g_last_error = "layer " + std::to_string(i) + ": " + g_last_error;
+            return rc;
+        }
+        in = out;
+    }
+    return MNN_OK;
+}
+
+int mnn_net_device_status(mnn_net_t net, void* stream, int* code, int* layer)
+{
+    if (!net || !code || !layer) return fail(MNN_EINVAL, "NULL argument");
+    *code = 0;
+    *layer = -1;
+    for (size_t i = 0; i < net->plans.size(); ++i) {
+        int c = 0;
+        int rc = mnn_conv_device_status(net->plans[i], stream, &c);
+        if (rc != MNN_OK) return rc;
+        if (c != 0 && *code == 0) {
+            *code = c;
+            *layer = (int)i;
+        }
+    }
+    return MNN_OK;
+}
+
+void mnn_net_destroy(mnn_net_t net) { delete net; }
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------
 // A run that allocates nothing: the plan's workspace is a fixed array that is
 // part of the library image on every GPU that loads it.
 // ---------------------------------------------------------------------------
@@ -592,6 +798,7 @@ extern "C" int mnn_conv_run_static(mnn_conv_plan_t p, const float* x, const floa
     local.prepared_w = nullptr;
     local.uc.ready = false;
     local.ws = nullptr;
+    local.tws = nullptr;
     local.ws_bytes = 0;
     if (local.workspace_bytes > 0) {
         void* ptr = nullptr;
