@@ -186,21 +186,25 @@ __global__ void __launch_bounds__(256) direct_generic_kernel(const float* __rest
 // enough loads in flight for the kernel to follow the memory system rather than its latency.
 constexpr int kDwBandRows = 32;   // output rows per unit
 
-template <int STRIDE>
+// SW = lanes per plane segment (32, 16 or 8): narrow planes put 2 or 4 channel planes side by side in a warp.
+template <int STRIDE, int SW>
 __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restrict__ x, const float* __restrict__ w,
                                                            const float* __restrict__ bias, float* __restrict__ y,
-                                                           DirectGeom g, int strips, int bands, long long n_units)
+                                                           DirectGeom g, int strips, int bands, long long n_planes,
+                                                           long long n_units)
 {
-    const int lane = threadIdx.x & 31;
-    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (plane, band, strip)
+    constexpr int PPW = 32 / SW;                      // planes per warp
+    const int lane = threadIdx.x & 31, ls = lane % SW, seg = lane / SW;
+    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (plane group, band, strip)
     if (unit >= n_units) return;
     const int strip = (int)(unit % strips);
     const long long rest = unit / strips;
     const int band = (int)(rest % bands);
-    const long long plane = rest / bands;
-    const int c = (int)(plane % g.Cout);
-    const float* xp = x + (size_t)plane * g.H * g.W;
-    float* yp = y + (size_t)plane * g.OH * g.OW;
+    const long long plane = (rest / bands) * PPW + seg;
+    const bool plane_ok = plane < n_planes;
+    const int c = (int)((plane_ok ? plane : 0) % g.Cout);
+    const float* xp = x + (size_t)(plane_ok ? plane : 0) * g.H * g.W;
+    float* yp = y + (size_t)(plane_ok ? plane : 0) * g.OH * g.OW;
     float wk[9];
 #pragma unroll
     for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + (size_t)c * 9 + i);
@@ -209,16 +213,22 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
     const unsigned full = 0xffffffffu;
 
     if (STRIDE == 1) {
-        // the 32 lanes hold input columns strip * 30 - 1 + lane; the 30 interior lanes produce outputs
-        const int iw = strip * 30 - 1 + lane;
+        // a segment holds input columns strip * (SW - 2) - 1 + ls; lanes 1 .. SW - 2 produce outputs, and so does
+        // the last lane when its right neighbour lies beyond the image (it is zero padding then)
+        const int iw = strip * (SW - 2) - 1 + ls;
         const int ow = iw;
-        const bool col_ok = iw >= 0 && iw < g.W;
-        const bool out_ok = lane >= 1 && lane <= 30 && ow < g.OW;
+        const bool col_ok = plane_ok && iw >= 0 && iw < g.W;
+        const bool last_edge = ls == SW - 1 && iw + 1 >= g.W;
+        const bool out_ok = col_ok && ls >= 1 && (ls <= SW - 2 || last_edge) && ow < g.OW;
         auto row = [&](int ih) { return (col_ok && ih >= 0 && ih < g.H) ? __ldg(xp + (size_t)ih * g.W + iw) : 0.0f; };
+        auto right = [&](float v) {
+            const float n = __shfl_down_sync(full, v, 1, SW);
+            return ls == SW - 1 ? 0.0f : n;
+        };
         // per input row: the lane's own value and its left / right neighbours (shuffled once, when the row arrives)
         float r0 = row(oh0 - 1), r1 = row(oh0);
-        float l0 = __shfl_up_sync(full, r0, 1), q0 = __shfl_down_sync(full, r0, 1);
-        float l1 = __shfl_up_sync(full, r1, 1), q1 = __shfl_down_sync(full, r1, 1);
+        float l0 = __shfl_up_sync(full, r0, 1, SW), q0 = right(r0);
+        float l1 = __shfl_up_sync(full, r1, 1, SW), q1 = right(r1);
         for (int oh = oh0; oh < oh1; oh += 4) {
             float nx[4];
 #pragma unroll
@@ -227,7 +237,7 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
             for (int k = 0; k < 4; ++k) {
                 if (oh + k < oh1) {
                     const float r2 = nx[k];
-                    const float l2 = __shfl_up_sync(full, r2, 1), q2 = __shfl_down_sync(full, r2, 1);
+                    const float l2 = __shfl_up_sync(full, r2, 1, SW), q2 = right(r2);
                     float acc = b;
                     acc = fmaf(wk[0], l0, acc); acc = fmaf(wk[1], r0, acc); acc = fmaf(wk[2], q0, acc);
                     acc = fmaf(wk[3], l1, acc); acc = fmaf(wk[4], r1, acc); acc = fmaf(wk[5], q1, acc);
@@ -239,12 +249,13 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
             }
         }
     } else {
-        // lane l produces output column ow = strip * 32 + l from input columns 2 ow - 1 + {0, 1, 2}: it loads the
-        // first two and takes the third from the next lane (the last lane loads its own)
-        const int ow = strip * 32 + lane;
+        // lane ls of a segment produces output column ow = strip * SW + ls from input columns 2 ow - 1 + {0, 1, 2}:
+        // it loads the first two and takes the third from the next lane (the segment's last lane loads its own)
+        const int ow = strip * SW + ls;
         const int iw0 = 2 * ow - 1;
-        const bool out_ok = ow < g.OW;
-        const bool c0_ok = iw0 >= 0 && iw0 < g.W, c1_ok = iw0 + 1 < g.W, c2_ok = lane == 31 && iw0 + 2 < g.W;
+        const bool out_ok = plane_ok && ow < g.OW;
+        const bool c0_ok = plane_ok && iw0 >= 0 && iw0 < g.W, c1_ok = plane_ok && iw0 + 1 < g.W,
+                   c2_ok = plane_ok && ls == SW - 1 && iw0 + 2 < g.W;
         struct Row { float v0, v1, v2; };
         auto load = [&](int ih, Row& r) {
             const bool ok = ih >= 0 && ih < g.H;
@@ -254,8 +265,8 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
             r.v2 = (ok && c2_ok) ? __ldg(p + 2) : 0.0f;
         };
         auto third = [&](Row& r) {
-            const float n = __shfl_down_sync(full, r.v0, 1);
-            if (lane != 31) r.v2 = n;
+            const float n = __shfl_down_sync(full, r.v0, 1, SW);
+            if (ls != SW - 1) r.v2 = n;
         };
         auto out = [&](int oh, const Row& a, const Row& m, const Row& z) {
             float acc = b;
@@ -313,15 +324,27 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
                             (g.stride == 1 || g.stride == 2);
     if (depthwise3) {
         const long long planes = (long long)g.N * g.Cout;
-        const int strips = g.stride == 1 ? (g.OW + 29) / 30 : (g.OW + 31) / 32;
+        // lanes per plane segment: a stride-1 segment of SW lanes covers SW - 1 input columns from -1 on, a
+        // stride-2 segment SW output columns
+        const int need = g.stride == 1 ? g.W + 1 : g.OW;
+        const int sw = need <= 8 ? 8 : (need <= 16 ? 16 : 32);
+        const int strips = sw < 32 ? 1 : (g.stride == 1 ? (g.OW + 29) / 30 : (g.OW + 31) / 32);
         const int bands = (g.OH + kDwBandRows - 1) / kDwBandRows;
-        const long long units = planes * strips * bands;
+        const long long groups = (planes + 32 / sw - 1) / (32 / sw);
+        const long long units = groups * strips * bands;
         const long long blocks = (units + 3) / 4;
         if (blocks > 2147483647ll) return cudaErrorInvalidValue;
-        if (g.stride == 1)
-            depthwise3x3_kernel<1><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, units);
-        else
-            depthwise3x3_kernel<2><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, units);
+#define MNNB_DW_LAUNCH(ST, SWV) depthwise3x3_kernel<ST, SWV><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, planes, units)
+        if (g.stride == 1) {
+            if (sw == 8) MNNB_DW_LAUNCH(1, 8);
+            else if (sw == 16) MNNB_DW_LAUNCH(1, 16);
+            else MNNB_DW_LAUNCH(1, 32);
+        } else {
+            if (sw == 8) MNNB_DW_LAUNCH(2, 8);
+            else if (sw == 16) MNNB_DW_LAUNCH(2, 16);
+            else MNNB_DW_LAUNCH(2, 32);
+        }
+#undef MNNB_DW_LAUNCH
         return cudaGetLastError();
     }
     long long blocks = (total + 255) / 256;
