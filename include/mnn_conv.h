@@ -231,7 +231,9 @@ MNN_API long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int
  * consts[4] attoseconds per fp32 ALU flop     consts[5] picoseconds of fixed cost per kernel (launch, ramp-up, tail)
  * consts[6] L2 bytes usable for one chunk     consts[7] number of SMs
  * consts[8] attoseconds per flop of the direct kernel
- * consts[9..15] reserved (0).
+ * consts[9] attoseconds per flop of the direct kernel for layers with at most 4 input channels
+ *           (0 = use consts[8])
+ * consts[10..15] reserved (0).
  * mnn_calibrate measures them on the current device (launches micro-benchmarks and
  * synchronises; allocates and frees its own scratch) and installs them;
  * mnn_set_calibration installs a frozen record so that plans are reproducible;

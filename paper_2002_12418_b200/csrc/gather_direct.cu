@@ -179,6 +179,63 @@ __global__ void __launch_bounds__(256) direct_generic_kernel(const float* __rest
     }
 }
 
+// Layers with very few input channels (network stems: Cin <= 4, groups 1): one thread per output pixel.  The
+// weights sit in shared memory as [tap][output channel], so the 32 output channels a thread accumulates at a
+// time come from eight broadcast 128-bit loads per tap; the patch values are re-read per group of 32 channels
+// from L1.  Stores are coalesced along the pixels.
+constexpr int kStemThreads = 128;
+constexpr int kStemCoChunk = 32;
+
+__global__ void __launch_bounds__(kStemThreads) direct_stem_kernel(const float* __restrict__ x, const float* __restrict__ w,
+                                                                   const float* __restrict__ bias, float* __restrict__ y,
+                                                                   DirectGeom g, int co_pad)
+{
+    extern __shared__ __align__(16) float s_w[];              // [Cin * k * k][co_pad]
+    const int taps = g.Cin * g.k * g.k;
+    for (int i = threadIdx.x; i < taps * co_pad; i += kStemThreads) {
+        const int tap = i / co_pad, co = i - tap * co_pad;
+        s_w[i] = co < g.Cout ? __ldg(w + (size_t)co * taps + tap) : 0.0f;
+    }
+    __syncthreads();
+    const int ohw = g.OH * g.OW;
+    const int n = blockIdx.y;
+    const int pix = blockIdx.x * kStemThreads + threadIdx.x;
+    if (pix >= ohw) return;
+    const int oh = pix / g.OW, ow = pix - oh * g.OW;
+    const int ih0 = oh * g.stride - g.pad, iw0 = ow * g.stride - g.pad;
+    const float* xn = x + (size_t)n * g.Cin * g.H * g.W;
+    float* yn = y + (size_t)n * g.Cout * ohw + pix;
+    for (int c0 = 0; c0 < g.Cout; c0 += kStemCoChunk) {
+        float acc[kStemCoChunk];
+#pragma unroll
+        for (int j = 0; j < kStemCoChunk; ++j) acc[j] = (bias && c0 + j < g.Cout) ? __ldg(bias + c0 + j) : 0.0f;
+        int tap = 0;
+        for (int ci = 0; ci < g.Cin; ++ci) {
+            const float* xc = xn + (size_t)ci * g.H * g.W;
+            for (int a = 0; a < g.k; ++a) {
+                const int ih = ih0 + a * g.dil;
+                const bool row_ok = ih >= 0 && ih < g.H;
+                for (int b = 0; b < g.k; ++b, ++tap) {
+                    const int iw = iw0 + b * g.dil;
+                    const float v = (row_ok && iw >= 0 && iw < g.W) ? __ldg(xc + (size_t)ih * g.W + iw) : 0.0f;
+                    const float4* wp = reinterpret_cast<const float4*>(s_w + (size_t)tap * co_pad + c0);
+#pragma unroll
+                    for (int q = 0; q < kStemCoChunk / 4; ++q) {
+                        const float4 w4 = wp[q];
+                        acc[4 * q] = fmaf(w4.x, v, acc[4 * q]);
+                        acc[4 * q + 1] = fmaf(w4.y, v, acc[4 * q + 1]);
+                        acc[4 * q + 2] = fmaf(w4.z, v, acc[4 * q + 2]);
+                        acc[4 * q + 3] = fmaf(w4.w, v, acc[4 * q + 3]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kStemCoChunk; ++j)
+            if (c0 + j < g.Cout) yn[(size_t)(c0 + j) * ohw] = g.relu ? fmaxf(acc[j], 0.0f) : acc[j];
+    }
+}
+
 // Depthwise 3x3 (groups = C, dilation 1, padding 1, stride 1 or 2): one warp sweeps a strip of one channel
 // plane downwards over a band of output rows.  A lane holds its column of the three input rows that an output
 // row needs; horizontal neighbours come from warp shuffles, so every input element is loaded once per strip
@@ -315,6 +372,12 @@ cudaError_t launch_gather(const float* x, void* V_hi, void* V_lo, const GatherGe
     return launch_overlapped(gather_kernel, dim3((unsigned)bx, (unsigned)by), dim3(256), 0, stream, x, V_hi, V_lo, g, T, mode);
 }
 
+bool direct_stem_applies(const DirectGeom& g)
+{
+    const long long smem = (long long)g.Cin * g.k * g.k * ((g.Cout + 31) / 32 * 32) * 4;
+    return g.groups == 1 && g.Cin <= 4 && g.N <= 65535 && smem <= 160 * 1024;
+}
+
 cudaError_t launch_direct(const float* x, const float* w, const float* bias, float* y, const DirectGeom& g,
                           cudaStream_t stream)
 {
@@ -345,6 +408,17 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
             else MNNB_DW_LAUNCH(2, 32);
         }
 #undef MNNB_DW_LAUNCH
+        return cudaGetLastError();
+    }
+    if (direct_stem_applies(g)) {
+        const int co_pad = (g.Cout + kStemCoChunk - 1) / kStemCoChunk * kStemCoChunk;
+        const size_t smem = (size_t)g.Cin * g.k * g.k * co_pad * sizeof(float);
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(direct_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        const dim3 grid((unsigned)((g.OH * g.OW + kStemThreads - 1) / kStemThreads), (unsigned)g.N);
+        direct_stem_kernel<<<grid, kStemThreads, smem, stream>>>(x, w, bias, y, g, co_pad);
         return cudaGetLastError();
     }
     long long blocks = (total + 255) / 256;

@@ -124,5 +124,7 @@ struct DirectGeom {
 };
 cudaError_t launch_direct(const float* x, const float* w, const float* bias, float* y, const DirectGeom& g,
                           cudaStream_t stream);
+// True when the direct path uses its kernel for layers with very few input channels (Cin <= 4, groups 1).
+bool direct_stem_applies(const DirectGeom& g);
 
 }  // namespace mnnb

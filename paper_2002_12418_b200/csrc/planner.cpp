@@ -46,6 +46,7 @@ Calibration default_calibration()
     c.c[6] = 80ll << 20;  // L2 bytes one chunk's V + M may occupy
     c.c[7] = 148;         // SMs
     c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
+    c.c[9] = 50000;       // as per flop of the direct kernel for Cin <= 4 (~20 TFLOP/s)
     return c;
 }
 
@@ -295,7 +296,11 @@ uint64_t direct_cost(const LayerShape& s, const Calibration& cal)
     const uint64_t y_bytes = 4ull * s.N * s.Cout * s.OH * s.OW;
     const uint64_t w_bytes = 4ull * s.Cout * (s.Cin / s.groups) * s.k * s.k;
     const uint64_t flops = 2ull * s.N * s.Cout * (s.Cin / s.groups) * s.OH * s.OW * s.k * s.k;
-    return kernel_ps((x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, flops * (uint64_t)cal.c[8], cal);
+    // layers with at most 4 input channels (groups 1) run a dedicated kernel with its own rate (consts[9])
+    const bool stem = s.groups == 1 && s.Cin <= 4 && cal.c[9] > 0 &&
+                      (long long)s.Cin * s.k * s.k * ((s.Cout + 31) / 32 * 32) * 4 <= 160 * 1024 && s.N <= 65535;
+    const uint64_t rate = (uint64_t)(stem ? cal.c[9] : cal.c[8]);
+    return kernel_ps((x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, flops * rate, cal);
 }
 
 uint64_t gemm_cost(const LayerShape& s, int operand, const Calibration& cal)
@@ -306,7 +311,10 @@ uint64_t gemm_cost(const LayerShape& s, int operand, const Calibration& cal)
     const uint64_t x_bytes = 4ull * s.N * s.Cin * s.H * s.W;
     const uint64_t y_bytes = 4ull * s.N * s.Cout * s.OH * s.OW;
     const uint64_t v_bytes = T * Kp * b, u_bytes = (uint64_t)s.Cout * Kp * b;
-    const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0], 0, 0, cal);
+    // the patch gather: a transposition at about two thirds of the copy rate for 1x1 stride-1 layers, a generic
+    // element-wise gather at about a fifth of it otherwise (measured)
+    const bool transposer = s.k == 1 && s.stride == 1 && s.pad == 0 && (s.H * s.W) % 4 == 0;
+    const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3 : 10) / 2, 0, 0, cal);
     const uint64_t contract = kernel_ps((v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0],
                                         2ull * T * s.Cout * Kp * tensor_as(operand, cal), 0, cal);
     return gather + contract;
