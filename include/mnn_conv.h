@@ -52,6 +52,7 @@ enum { MNN_ALGO_AUTO = 0, MNN_ALGO_WINOGRAD = 1, MNN_ALGO_GEMM = 2, MNN_ALGO_DIR
 enum { MNN_PREC_TF32 = 0, MNN_PREC_BF16 = 1 };             /* accuracy class */
 enum { MNN_OPERAND_AUTO = 0, MNN_OPERAND_TF32 = 1, MNN_OPERAND_BF16 = 2, MNN_OPERAND_FP32_REF = 3 };
 enum { MNN_POINTS_AUTO = 0, MNN_POINTS_PAPER = 1, MNN_POINTS_UNIT = 2, MNN_POINTS_MIXED = 3 };
+enum { MNN_GEMM_LHS_AUTO = 0, MNN_GEMM_LHS_PATCHES = 1, MNN_GEMM_LHS_X = 2 };
 enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_STAGE_OUTPUT = 8,
        MNN_STAGE_ALL = 15 };
 
@@ -81,6 +82,14 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
  *   chunk_images  0 = planner; else images per pipeline chunk.  The planner cuts the
  *              batch only when the transformed tensors of the whole batch would
  *              exceed 4 GiB.
+ *   gemm_lhs   left operand of the GEMM scheme.  PATCHES: the gathered patch matrix
+ *              V [N*OH*OW][Cin*k*k] in the operand format.  X: the input itself, read as
+ *              the pixel-contiguous matrix [Cin][H*W] of each image (no gather, no V);
+ *              only for 1x1 stride-1 unpadded ungrouped layers with H*W >= 32 and a
+ *              multiple of 4 and single-pass TF32 operands, where the tensor core drops
+ *              the low 13 mantissa bits of x (truncation) instead of a rounded copy being
+ *              stored.  AUTO = the planner takes the cheaper where X applies.  Asking
+ *              for X where it does not apply fails the plan.
  */
 typedef struct {
     int groups;
@@ -92,7 +101,8 @@ typedef struct {
     int force_m;
     int points_id;
     int chunk_images;
-    int reserved[7];
+    int gemm_lhs;
+    int reserved[6];
 } mnn_conv_opts;
 
 /*
@@ -118,7 +128,7 @@ typedef struct {
     long long u_offset, u_bytes, v_offset, v_bytes, m_offset, m_bytes;
     long long predicted_error_ppm;   /* accuracy model's relative L2 error x 1e6 for the choice */
     int chosen_candidate;            /* index into cost_ps, -1 when the choice was forced outside the list */
-    int reserved;
+    int gemm_lhs;                    /* GEMM scheme: MNN_GEMM_LHS_PATCHES or MNN_GEMM_LHS_X as planned, else 0 */
     unsigned long long cost_ps[MNN_N_CANDIDATES];
 } mnn_conv_info;
 

@@ -47,6 +47,7 @@ struct mnn_conv_plan_s {
     int m_row_stride = 0;
     long long u_offset = 0, u_bytes = 0, v_offset = 0, v_bytes = 0, m_offset = 0, m_bytes = 0, workspace_bytes = 0;
     int launches_per_run = 1;
+    bool gemm_x = false;             // GEMM scheme with x itself as the left operand: no V, one launch
     TransformMatrices mats;
     // run-time state
     char* ws = nullptr;              // status word and U (persistent part), and V, M unless tws is set
@@ -107,9 +108,10 @@ void layout_workspace(mnn_conv_plan_t p)
         p->chunk_tiles = (long long)s.N * s.OH * s.OW;
         p->m_row_stride = 0;
         p->u_bytes = align_up((long long)s.Cout * p->cin_pad * eb, 2048);
-        p->v_bytes = align_up(p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->gemm_x = d.gemm_lhs == MNN_GEMM_LHS_X;
+        p->v_bytes = p->gemm_x ? 0 : align_up(p->chunk_tiles * p->cin_pad * eb, 2048);
         p->m_bytes = 0;
-        p->launches_per_run = 2;
+        p->launches_per_run = p->gemm_x ? 1 : 2;
     }
     p->u_offset = off;
     off += p->u_bytes;
@@ -271,6 +273,7 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     info->m_bytes = p->m_bytes;
     info->predicted_error_ppm = p->d.error_ppm;
     info->chosen_candidate = p->d.chosen;
+    info->gemm_lhs = p->d.algo == MNN_ALGO_GEMM ? p->d.gemm_lhs : 0;
     for (int i = 0; i < MNN_N_CANDIDATES; ++i) info->cost_ps[i] = p->d.cost_ps[i];
     return MNN_OK;
 }
@@ -327,8 +330,11 @@ static int set_workspace_split(mnn_conv_plan_t p, void* persistent, long long pe
     if (p->d.operand != MNN_OPERAND_FP32_REF) {
         const char* why = "";
         const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
-        e = umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p),
-                                v_hi(p), v_lo(p), &why);
+        if (p->gemm_x)
+            e = umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), &why);
+        else
+            e = umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p),
+                                    v_hi(p), v_lo(p), &why);
         if (e != cudaSuccess) {
             p->ws = nullptr;
             return fail(MNN_ECUDA, std::string("tensor-core contraction setup: ") + why + " (" + cudaGetErrorString(e) + ")");
@@ -343,7 +349,7 @@ static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, con
     if ((mask & ~(unsigned)MNN_STAGE_ALL) || mask == 0) return fail(MNN_EINVAL, "bad stage mask");
     if (p->workspace_bytes > 0 && !p->ws) return fail(MNN_EWORKSPACE, "call mnn_conv_set_workspace first");
     const bool direct = p->d.algo == MNN_ALGO_DIRECT;
-    const bool need_x = direct || (mask & MNN_STAGE_INPUT);
+    const bool need_x = direct || (mask & MNN_STAGE_INPUT) || (p->gemm_x && (mask & MNN_STAGE_CONTRACT));
     const bool need_w = direct || (mask & MNN_STAGE_WEIGHT);
     const bool need_y = direct || (mask & MNN_STAGE_OUTPUT) || (p->d.algo == MNN_ALGO_GEMM && (mask & MNN_STAGE_CONTRACT));
     if ((need_x && !x) || (need_w && !w) || (need_y && !y)) return fail(MNN_EINVAL, "NULL tensor pointer");
@@ -409,7 +415,7 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
 
     if (d.algo == MNN_ALGO_GEMM) {
         const long long T = (long long)s.N * s.OH * s.OW;
-        if (mask & MNN_STAGE_INPUT) {
+        if ((mask & MNN_STAGE_INPUT) && !p->gemm_x) {
             GatherGeom g = {s.N, s.Cin, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, p->cin_pad};
             LaunchTimer lt(p, st, 1);
             e = launch_gather(x, v_hi(p), v_lo(p), g, p->store_mode, st);
@@ -421,6 +427,8 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
             if (reference)
                 e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, 1, s.Cout, T, p->cin_pad,
                                               (long long)s.Cout * p->cin_pad, T * p->cin_pad, epi, st);
+            else if (p->gemm_x)
+                e = launch_contract_umma_x(p->uc, x, epi, status_word(p), st);
             else
                 e = launch_contract_umma(p->uc, T, epi, status_word(p), st);
             if (e != cudaSuccess) return fail_cuda(e, "GEMM contraction");
@@ -812,8 +820,12 @@ extern "C" int mnn_conv_run_static(mnn_conv_plan_t p, const float* x, const floa
         if (local.d.operand != MNN_OPERAND_FP32_REF) {
             const char* why = "";
             const int alpha2 = local.d.algo == MNN_ALGO_WINOGRAD ? local.d.alpha * local.d.alpha : 1;
-            e = umma_contract_setup(&local.uc, local.store_mode, alpha2, local.s.Cout, local.cin_pad, local.chunk_tiles,
-                                    u_hi(&local), u_lo(&local), v_hi(&local), v_lo(&local), &why);
+            if (local.gemm_x)
+                e = umma_contract_setup_x(&local.uc, local.s.Cout, local.s.Cin, local.cin_pad, local.s.N,
+                                          local.s.H * local.s.W, u_hi(&local), &why);
+            else
+                e = umma_contract_setup(&local.uc, local.store_mode, alpha2, local.s.Cout, local.cin_pad, local.chunk_tiles,
+                                        u_hi(&local), u_lo(&local), v_hi(&local), v_lo(&local), &why);
             if (e != cudaSuccess)
                 return fail(MNN_ECUDA, std::string("tensor-core contraction setup: ") + why + " (" + cudaGetErrorString(e) + ")");
         }

@@ -5,7 +5,10 @@
 // A persistent, warp-specialised kernel: one thread feeds shared memory with TMA
 // (128-byte-swizzled K-major tiles of V and U), one thread issues tcgen05.mma with
 // the accumulator in tensor memory (128 tiles x BN output channels, double
-// buffered), four warps drain the accumulator with tcgen05.ld and store it.
+// buffered), four warps drain the accumulator with tcgen05.ld and store it (one per
+// quarter of the tensor-memory lanes, the load of the next 16 columns in flight while
+// the previous 16 are stored; two warps per quarter, each taking half of the columns,
+// were measured and gained nothing: the stores already run near the HBM write rate).
 // The MMA "M" dimension is the tile index t (operand A = V), "N" the output channel
 // (operand B = U), "K" the input channel; TF32 or BF16 operands, fp32 accumulation;
 // with passes = 3 the operands come as hi + lo pairs and hi*hi + lo*hi + hi*lo are
@@ -14,16 +17,24 @@
 // store: one full line per request.  (With channels on the lanes and 128-bit stores
 // the instruction count is lower but every store touches 32 rows; measured slower on
 // short K loops, where the epilogue decides.)
+//
+// A 1x1 stride-1 convolution needs no patch matrix: x[n] = [Cin][H*W] already is operand A, stored with the
+// M index (the pixel) contiguous.  In that mode (a_mn) the producer copies boxes of 32 pixels x 32 channels
+// straight out of x, the MMA reads A as an MN-major operand, and a work item covers four such 32-pixel
+// "atoms" (each inside one image), one per epilogue warp.  The tensor core drops the low 13 mantissa bits of
+// the fp32 values it is given (truncation, where the stored operands are rounded to nearest).
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "planner.h"
 #include "umma.cuh"
 
 namespace mnnb {
 
 namespace {
 
-constexpr int kThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kEpilogueWarps = 4;      // a multiple of 4: warps per quarter of the lanes split the columns
+constexpr int kThreads = 64 + 32 * kEpilogueWarps;   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
 constexpr int kTileM = 128;            // tiles (rows of V) per work item
 constexpr int kMaxStages = 8;
 constexpr int kMaxSharedBias = 2048;    // output channels whose bias is staged in shared memory (+ 16 of slack)
@@ -37,6 +48,9 @@ struct KernelParams {
     long long n_items;
     ContractEpilogue epi;
     int* status;
+    // a_mn mode: operand A comes from x [images][Cin][hw]; 32-pixel atoms, atoms_per_image = ceil(hw / 32)
+    int a_mn, hw, atoms_per_image;
+    long long total_atoms;
 };
 
 // status codes written on a bounded wait that ran out
@@ -74,7 +88,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(ptx::smem_u32(&tfull_bar[s]), 1);
-            ptx::mbar_init(ptx::smem_u32(&tempty_bar[s]), 4);
+            ptx::mbar_init(ptx::smem_u32(&tempty_bar[s]), kEpilogueWarps);
         }
         abort_flag = 0;
         ptx::fence_barrier_init();
@@ -94,7 +108,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     const bool bias_in_smem = p.epi.mode == 1 && p.Cout <= kMaxSharedBias;
     if (bias_in_smem && warp >= 2) {
         for (int i = threadIdx.x - 64; i < p.Cout; i += kThreads - 64) s_bias[i] = p.epi.bias ? __ldg(p.epi.bias + i) : 0.0f;
-        asm volatile("bar.sync 1, 128;" ::: "memory");          // the four epilogue warps only
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");          // the epilogue warps only
     }
 
     const int k_elems = KIND == 0 ? 32 : 64;         // elements of K per 128-byte row
@@ -118,7 +132,17 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
                     const uint32_t sbase = smem_base + stage * stage_bytes;
                     ptx::mbar_expect_tx(bar, stage_bytes);
-                    ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
+                    if (p.a_mn) {
+#pragma unroll
+                        for (int j = 0; j < kTileM / 32; ++j) {
+                            // an atom past the end names an image that does not exist and reads as zeros
+                            const long long a = (long long)tb * (kTileM / 32) + j;
+                            const int img = (int)(a / p.atoms_per_image);
+                            const int pix0 = (int)(a - (long long)img * p.atoms_per_image) * 32;
+                            ptx::tma_load_3d(sbase + j * 4096, &map_v_hi, bar, pix0, kb * k_elems, img);
+                        }
+                    } else
+                        ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
                     ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
                     if (split == 2) {
                         ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM, xi);
@@ -133,7 +157,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = ptx::mma_idesc(KIND == 0 ? 2 : 1, kTileM, p.bn);
+            const uint32_t idesc = ptx::mma_idesc(KIND == 0 ? 2 : 1, kTileM, p.bn, p.a_mn != 0);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             for (long long item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
@@ -156,7 +180,9 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     const uint32_t sbase = smem_base + stage * stage_bytes;
 #pragma unroll
                     for (int ks = 0; ks < kSwizzleBytes / 32; ++ks) {
-                        const uint64_t a_hi = ptx::smem_desc_k128(sbase + ks * 32);
+                        // K-major: 8 K elements are 32 bytes along the row; MN-major: 8 rows of 128 bytes
+                        const uint64_t a_hi = p.a_mn ? ptx::smem_desc_mn128_b32(sbase + ks * 1024, 4096)
+                                                     : ptx::smem_desc_k128(sbase + ks * 32);
                         const uint64_t b_hi = ptx::smem_desc_k128(sbase + off_b_hi + ks * 32);
                         ptx::mma_ss<KIND>(d_tmem, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
                         if (split == 2) {
@@ -180,6 +206,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
         }
     } else {
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int part = (warp - 2) >> 2;             // which part of the columns this warp drains
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         for (long long item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
@@ -201,7 +228,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
             }
             ptx::tc_fence_after();
             const long long t = (long long)tb * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
-            const bool t_ok = t < p.tiles;
+            bool t_ok = t < p.tiles;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)p.bn;
             const int co0 = nb * p.bn;
             const int n_co = min(p.bn, p.Cout - co0);                        // valid output channels of this item
@@ -211,65 +238,88 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
             if (p.epi.mode == 0) {
                 step = p.epi.m_row_stride;
                 dst = p.epi.M + ((size_t)xi * p.Cout + co0) * p.epi.m_row_stride + t;
+            } else if (p.a_mn) {
+                const long long a = (long long)tb * (kTileM / 32) + q;       // this warp's atom
+                const long long img = a / p.atoms_per_image;
+                const int pix = (int)(a - img * p.atoms_per_image) * 32 + lane;
+                t_ok = a < p.total_atoms && pix < p.hw;
+                step = p.hw;
+                dst = p.epi.y + ((size_t)(t_ok ? img : 0) * p.Cout + co0) * p.hw + (t_ok ? pix : 0);
             } else {
                 const long long img = t_ok ? t / p.epi.ohw : 0;
                 step = p.epi.ohw;
                 dst = p.epi.y + ((size_t)img * p.Cout + co0) * p.epi.ohw + (t_ok ? t - img * p.epi.ohw : 0);
             }
-            for (int c0 = 0; c0 < n_co; c0 += 16) {
-                uint32_t v[16];
-                ptx::tmem_ld16(taddr + (uint32_t)c0, v);
-                ptx::tmem_ld_wait();
-                if (t_ok) {
-                    const int n = min(16, n_co - c0);
-                    float* pj = dst;                                   // walks the 16 channels of this chunk
-                    if (p.epi.mode == 0) {
-                        if (n == 16) {
+            // this warp's chunks of 16 columns
+            constexpr int kParts = kEpilogueWarps / 4;
+            const int n_chunks = (n_co + 15) >> 4;
+            const int per_part = (n_chunks + kParts - 1) / kParts;
+            const int ch_begin = min(part * per_part, n_chunks), ch_end = min(ch_begin + per_part, n_chunks);
+            dst += (long long)ch_begin * 16 * step;
+            const bool relu = p.epi.relu != 0;
+            auto store_chunk = [&](const uint32_t (&v)[16], int ch) {
+                if (!t_ok) return;
+                const int c0 = ch * 16;
+                const int n = min(16, n_co - c0);
+                float* pj = dst;                                   // walks the 16 channels of this chunk
+                if (p.epi.mode == 0) {
+                    if (n == 16) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                *pj = __uint_as_float(v[j]);
-                                pj += step;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                if (j < n) *pj = __uint_as_float(v[j]);
-                                pj += step;
-                            }
+                        for (int j = 0; j < 16; ++j) {
+                            *pj = __uint_as_float(v[j]);
+                            pj += step;
                         }
                     } else {
-                        float bz[16];
-                        if (bias_in_smem) {
-                            // (reads past Cout stay inside the array and are not used)
-                            const float4* bp = reinterpret_cast<const float4*>(s_bias + co0 + c0);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float4 q4 = bp[j];
-                                bz[4 * j] = q4.x; bz[4 * j + 1] = q4.y; bz[4 * j + 2] = q4.z; bz[4 * j + 3] = q4.w;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) bz[j] = (p.epi.bias && j < n) ? __ldg(p.epi.bias + co0 + c0 + j) : 0.0f;
+                        for (int j = 0; j < 16; ++j) {
+                            if (j < n) *pj = __uint_as_float(v[j]);
+                            pj += step;
                         }
-                        const bool relu = p.epi.relu != 0;
-                        if (n == 16) {
+                    }
+                } else {
+                    float bz[16];
+                    if (bias_in_smem) {
+                        // (reads past Cout stay inside the array and are not used)
+                        const float4* bp = reinterpret_cast<const float4*>(s_bias + co0 + c0);
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const float o = __uint_as_float(v[j]) + bz[j];
-                                *pj = relu ? fmaxf(o, 0.0f) : o;
-                                pj += step;
-                            }
-                        } else {
+                        for (int j = 0; j < 4; ++j) {
+                            const float4 q4 = bp[j];
+                            bz[4 * j] = q4.x; bz[4 * j + 1] = q4.y; bz[4 * j + 2] = q4.z; bz[4 * j + 3] = q4.w;
+                        }
+                    } else {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const float o = __uint_as_float(v[j]) + bz[j];
-                                if (j < n) *pj = relu ? fmaxf(o, 0.0f) : o;
-                                pj += step;
-                            }
+                        for (int j = 0; j < 16; ++j) bz[j] = (p.epi.bias && j < n) ? __ldg(p.epi.bias + co0 + c0 + j) : 0.0f;
+                    }
+                    if (n == 16) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float o = __uint_as_float(v[j]) + bz[j];
+                            *pj = relu ? fmaxf(o, 0.0f) : o;
+                            pj += step;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float o = __uint_as_float(v[j]) + bz[j];
+                            if (j < n) *pj = relu ? fmaxf(o, 0.0f) : o;
+                            pj += step;
                         }
                     }
                 }
+            };
+            uint32_t va[16], vb[16];
+            if (ch_begin < ch_end) ptx::tmem_ld16(taddr + (uint32_t)(ch_begin * 16), va);
+            for (int ch = ch_begin; ch < ch_end; ch += 2) {
+                ptx::tmem_ld_wait();
+                if (ch + 1 < ch_end) ptx::tmem_ld16(taddr + (uint32_t)((ch + 1) * 16), vb);
+                store_chunk(va, ch);
                 dst += 16 * step;
+                if (ch + 1 < ch_end) {
+                    ptx::tmem_ld_wait();
+                    if (ch + 2 < ch_end) ptx::tmem_ld16(taddr + (uint32_t)((ch + 2) * 16), va);
+                    store_chunk(vb, ch + 1);
+                    dst += 16 * step;
+                }
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -365,6 +415,11 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
                                 void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why)
 {
     uc->ready = false;
+    uc->a_mn = V_hi == nullptr;        // operand A is read from x at launch time (umma_contract_setup_x)
+    if (uc->a_mn && (mode != STORE_TF32 || alpha2 != 1)) {
+        *why = "reading x as operand A needs single-pass TF32 and one transform position";
+        return cudaErrorInvalidValue;
+    }
     if (mode == STORE_FP32) {
         *why = "the tensor-core contraction needs TF32 or BF16 operands";
         return cudaErrorInvalidValue;
@@ -385,31 +440,8 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&uc->num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    // Output channels per work item (MMA N): a multiple of 16, at most 256, channel blocks balanced.  Wider
-    // blocks re-use the V tile more; narrower ones give more work items.  Among 1x, 2x and 4x the minimum
-    // number of blocks take the one with the shortest schedule: rounds of work items over the SMs times the
-    // operand rows an item loads (128 tiles + bn channels).  (Weighing the tensor side in as well was tried
-    // and measured slower on the 512-channel 14 x 14 layers.)
-    {
-        const int co16 = (Cout + 15) / 16 * 16;
-        const int min_blocks = (co16 + 255) / 256;
-        const long long tile_blocks = (tiles_capacity + kTileM - 1) / kTileM;
-        long long best_cost = -1;
-        for (int mult = 1; mult <= 4; mult *= 2) {
-            const int blocks = min_blocks * mult;
-            const int bn = ((co16 / 16 + blocks - 1) / blocks) * 16;
-            if (bn < 32 && mult > 1) break;
-            const int real_blocks = (co16 + bn - 1) / bn;
-            const long long items = tile_blocks * real_blocks * alpha2;
-            const long long rounds = (items + uc->num_sms - 1) / uc->num_sms;
-            const long long cost = rounds * (kTileM + bn);
-            if (best_cost < 0 || cost < best_cost) {
-                best_cost = cost;
-                uc->bn = bn;
-                uc->n_co_blocks = real_blocks;
-            }
-        }
-    }
+    // output channels per work item (MMA N) and the channel blocks
+    contract_tiling((tiles_capacity + kTileM - 1) / kTileM, alpha2, Cout, uc->num_sms, &uc->bn, &uc->n_co_blocks);
     const int k_elems = kSwizzleBytes / eb;
     uc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
     const int split = uc->passes == 3 ? 2 : 1;
@@ -429,7 +461,7 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     uc->tmem_cols = cols;
 
     const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
-    bool ok = encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
+    bool ok = (uc->a_mn || encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM)) &&
               encode_operand_map(&uc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
     if (ok && split == 2)
         ok = encode_operand_map(&uc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
@@ -438,6 +470,7 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
         *why = "cuTensorMapEncodeTiled failed or is unavailable";
         return cudaErrorInvalidValue;
     }
+    if (uc->a_mn) uc->map_v_hi = uc->map_u_hi;      // replaced by the map over x at every launch
     if (split == 1) {
         uc->map_v_lo = uc->map_v_hi;
         uc->map_u_lo = uc->map_u_hi;
@@ -452,13 +485,73 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     return cudaSuccess;
 }
 
+cudaError_t umma_contract_setup_x(UmmaContract* uc, int Cout, int Cin, int cin_pad, int images, int hw, void* U,
+                                  const char** why)
+{
+    if (hw < 32 || hw % 4 != 0) {
+        *why = "reading x as operand A needs H*W >= 32 and a multiple of 4";
+        return cudaErrorInvalidValue;
+    }
+    const long long atoms = (long long)images * ((hw + 31) / 32);
+    cudaError_t e = umma_contract_setup(uc, STORE_TF32, 1, Cout, cin_pad, atoms * 32, U, nullptr, nullptr, nullptr, why);
+    if (e != cudaSuccess) return e;
+    uc->x_images = images;
+    uc->x_cin = Cin;
+    uc->x_hw = hw;
+    uc->k_blocks = (Cin + 31) / 32;
+    return cudaSuccess;
+}
+
+cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const ContractEpilogue& epi, int* status,
+                                   cudaStream_t stream)
+{
+    if (!uc.ready || !uc.a_mn) return cudaErrorInvalidValue;
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return cudaErrorInvalidValue;
+    // x as [images][Cin][hw], box = 32 pixels x 32 channels of one image, 128-byte swizzle with a 32-byte base
+    CUtensorMap map_x;
+    const cuuint64_t dims[3] = {(cuuint64_t)uc.x_hw, (cuuint64_t)uc.x_cin, (cuuint64_t)uc.x_images};
+    const cuuint64_t strides[2] = {(cuuint64_t)uc.x_hw * 4, (cuuint64_t)uc.x_cin * uc.x_hw * 4};
+    const cuuint32_t box[3] = {32, 32, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (fn(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(x), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    KernelParams p;
+    p.a_mn = 1;
+    p.hw = uc.x_hw;
+    p.atoms_per_image = (uc.x_hw + 31) / 32;
+    p.total_atoms = (long long)uc.x_images * p.atoms_per_image;
+    p.alpha2 = 1;
+    p.n_tile_blocks = (int)((p.total_atoms + kTileM / 32 - 1) / (kTileM / 32));
+    p.n_co_blocks = uc.n_co_blocks;
+    p.bn = uc.bn;
+    p.k_blocks = uc.k_blocks;
+    p.passes = 1;
+    p.stages = uc.stages;
+    p.tmem_cols = uc.tmem_cols;
+    p.Cout = uc.Cout;
+    p.tiles = p.total_atoms * 32;
+    p.n_items = (long long)p.n_tile_blocks * p.n_co_blocks;
+    p.epi = epi;
+    p.status = status;
+    const long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
+    return launch_overlapped(contract_umma_kernel<0>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
+                             map_x, map_x, uc.map_u_hi, uc.map_u_lo, p);
+}
+
 cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const ContractEpilogue& epi, int* status,
                                  cudaStream_t stream)
 {
-    if (!uc.ready) return cudaErrorInvalidValue;
+    if (!uc.ready || uc.a_mn) return cudaErrorInvalidValue;
     if (tiles <= 0) return cudaSuccess;
     if (tiles > uc.tiles_capacity) return cudaErrorInvalidValue;
     KernelParams p;
+    p.a_mn = 0;
+    p.hw = 0;
+    p.atoms_per_image = 1;
+    p.total_atoms = 0;
     p.alpha2 = uc.alpha2;
     p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
     p.n_co_blocks = uc.n_co_blocks;

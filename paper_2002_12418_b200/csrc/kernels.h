@@ -109,6 +109,8 @@ struct UmmaContract {
     int tmem_cols;
     int smem_bytes;
     int num_sms;
+    bool a_mn = false;                 // operand A is x itself (1x1 stride-1 convolution), see umma_contract_setup_x
+    int x_images = 0, x_cin = 0, x_hw = 0;
     bool ready = false;
 };
 // Encodes the tensor maps for U/V at the given device addresses.  Returns a CUDA error or cudaSuccess;
@@ -117,6 +119,12 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
                                 void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why);
 cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const ContractEpilogue& epi, int* status,
                                  cudaStream_t stream);
+// 1x1 stride-1 unpadded convolution without a patch matrix: operand A is x [images][Cin][hw] (hw >= 32, a
+// multiple of 4, x 16-byte aligned), operand B is U [Cout][cin_pad] in TF32; epi.mode must be 1.
+cudaError_t umma_contract_setup_x(UmmaContract* uc, int Cout, int Cin, int cin_pad, int images, int hw, void* U,
+                                  const char** why);
+cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const ContractEpilogue& epi, int* status,
+                                   cudaStream_t stream);
 
 // Direct ("sliding window") convolution, any stride / padding / dilation / groups.
 struct DirectGeom {

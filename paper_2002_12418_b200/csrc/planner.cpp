@@ -303,7 +303,38 @@ uint64_t direct_cost(const LayerShape& s, const Calibration& cal)
     return kernel_ps((x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, flops * rate, cal);
 }
 
-uint64_t gemm_cost(const LayerShape& s, int operand, const Calibration& cal)
+}  // namespace
+
+void contract_tiling(long long tile_blocks, int alpha2, int Cout, int num_sms, int* bn_out, int* n_co_blocks)
+{
+    const int co16 = (Cout + 15) / 16 * 16;
+    const int min_blocks = (co16 + 255) / 256;
+    long long best_cost = -1;
+    for (int mult = 1; mult <= 4; mult *= 2) {
+        const int blocks = min_blocks * mult;
+        const int bn = ((co16 / 16 + blocks - 1) / blocks) * 16;
+        if (bn < 32 && mult > 1) break;
+        const int real_blocks = (co16 + bn - 1) / bn;
+        const long long items = tile_blocks * real_blocks * alpha2;
+        const long long rounds = (items + num_sms - 1) / num_sms;
+        const long long cost = rounds * (128 + bn);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            *bn_out = bn;
+            *n_co_blocks = real_blocks;
+        }
+    }
+}
+
+bool gemm_reads_x(const LayerShape& s, int operand, int passes)
+{
+    return s.k == 1 && s.stride == 1 && s.pad == 0 && s.groups == 1 && operand == MNN_OPERAND_TF32 && passes == 1 &&
+           s.H * s.W >= 32 && (s.H * s.W) % 4 == 0;
+}
+
+namespace {
+
+uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibration& cal)
 {
     const uint64_t b = operand_bytes(operand);
     const uint64_t Kp = round_up((uint64_t)s.Cin * s.k * s.k, 8);
@@ -315,8 +346,20 @@ uint64_t gemm_cost(const LayerShape& s, int operand, const Calibration& cal)
     // element-wise gather at about a fifth of it otherwise (measured)
     const bool transposer = s.k == 1 && s.stride == 1 && s.pad == 0 && (s.H * s.W) % 4 == 0;
     const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3 : 10) / 2, 0, 0, cal);
-    const uint64_t contract = kernel_ps((v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0],
-                                        2ull * T * s.Cout * Kp * tensor_as(operand, cal), 0, cal);
+    // The contraction as the kernel schedules it: rounds of work items over the SMs, each item a serial loop
+    // over blocks of K whose pace is the slower of the tensor core and the delivery of the two operand tiles
+    // from L2 to one SM (about 63 GB/s measured; about 21 GB/s for the pixel-contiguous tile read out of x).
+    const int sms = cal.c[7] > 0 ? (int)cal.c[7] : 148;
+    const uint64_t tile_blocks = lhs_x ? ceil_div((uint64_t)s.N * ceil_div((uint64_t)s.H * s.W, 32), 4) : ceil_div(T, 128);
+    int bn = 256, n_co_blocks = 1;
+    contract_tiling((long long)tile_blocks, 1, s.Cout, sms, &bn, &n_co_blocks);
+    const uint64_t rounds = ceil_div(tile_blocks * (uint64_t)n_co_blocks, (uint64_t)sms);
+    const uint64_t k_elems = 128 / b, k_blocks = ceil_div(Kp, k_elems);
+    const uint64_t deliver_ps = 128ull * 128 * (lhs_x ? 46 : 16) + (uint64_t)bn * 128 * 16;
+    const uint64_t mma_ps = 2ull * 128 * bn * k_elems * tensor_as(operand, cal) * sms / 1000000ull;
+    const uint64_t serial_as = rounds * k_blocks * (deliver_ps > mma_ps ? deliver_ps : mma_ps) * 1000000ull;
+    if (lhs_x) return kernel_ps((x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
+    const uint64_t contract = kernel_ps((v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
     return gather + contract;
 }
 
@@ -396,6 +439,7 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
     cands[15] = {0, 0, 0, 0};
 
     int chunk_of[MNN_N_CANDIDATES] = {0}, nch_of[MNN_N_CANDIDATES] = {0}, pts_of[MNN_N_CANDIDATES] = {0};
+    int lhs_of[MNN_N_CANDIDATES] = {0};
     long long ppm_of[MNN_N_CANDIDATES] = {0};
 
     for (int i = 0; i < 15; ++i) {
@@ -414,8 +458,16 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
             long long ppm = accuracy_ppm(1, s.k, 0, c.operand, c.passes);
             if (ppm < 0) continue;
             if ((uint64_t)ppm > gate_ppm && !(o.operand != 0 && o.force_algo == MNN_ALGO_GEMM)) continue;
+            // left operand: the patch matrix, or x itself where that applies (whichever is cheaper)
+            const bool x_ok = gemm_reads_x(s, c.operand, c.passes);
+            if (o.gemm_lhs == MNN_GEMM_LHS_X && !x_ok) continue;
+            const uint64_t cost_patches = gemm_cost(s, c.operand, false, cal);
+            const uint64_t cost_x = x_ok ? gemm_cost(s, c.operand, true, cal) : MNN_COST_INADMISSIBLE;
+            const bool take_x = o.gemm_lhs == MNN_GEMM_LHS_X || (o.gemm_lhs == MNN_GEMM_LHS_AUTO && x_ok && cost_x < cost_patches);
+            if (take_x && ppm < kGemmLhsXErrorPpm) ppm = kGemmLhsXErrorPpm;
+            lhs_of[i] = take_x ? MNN_GEMM_LHS_X : MNN_GEMM_LHS_PATCHES;
             ppm_of[i] = ppm;
-            d->cost_ps[i] = gemm_cost(s, c.operand, cal);
+            d->cost_ps[i] = take_x ? cost_x : cost_patches;
             continue;
         }
         // Winograd
@@ -466,6 +518,7 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
                 return MNN_EUNSUPPORTED;
             }
             d->algo = MNN_ALGO_GEMM;
+            d->gemm_lhs = MNN_GEMM_LHS_PATCHES;
             d->m = 1;
             d->alpha = 1;
             d->operand = MNN_OPERAND_FP32_REF;
@@ -509,6 +562,7 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
         d->points_id = 0;
         d->chunk_images = s.N;
         d->n_chunks = 1;
+        d->gemm_lhs = c.algo == MNN_ALGO_GEMM ? lhs_of[best] : 0;
     }
     return MNN_OK;
 }

@@ -163,11 +163,29 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t smem_addr)
     return d;
 }
 
-// Instruction descriptor: fp32 accumulate, both operands K-major, format 2 = TF32, 1 = BF16.
-__host__ __device__ constexpr uint32_t mma_idesc(int fmt, int M, int N)
+// Shared-memory matrix descriptor for an MN-major operand tile of 32-bit elements.  The tensor core takes such
+// operands only in the "128-byte swizzle with a 32-byte base": rows of 128 bytes hold 32 consecutive M (or N)
+// elements of one K index, and the four 32-byte pieces of a row are permuted by the row index modulo 4 (what
+// a TMA load with SWIZZLE_128B_ATOM_32B of a box {32 elements of M, rows of K} produces).  Four rows (512
+// bytes) form a swizzle atom; consecutive atoms along K are 512 bytes apart (stride byte offset) and the atoms
+// of consecutive 32-element groups of M `atom_stride_bytes` apart (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn128_b32(uint32_t smem_addr, uint32_t atom_stride_bytes)
 {
-    return (1u << 4) | ((uint32_t)fmt << 7) | ((uint32_t)fmt << 10) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((atom_stride_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(512 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)1 << 61;                                  // 128-byte swizzle, 32-byte base
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulate, format 2 = TF32, 1 = BF16; operand B K-major, operand A K-major
+// unless a_mn_major.
+__host__ __device__ constexpr uint32_t mma_idesc(int fmt, int M, int N, bool a_mn_major = false)
+{
+    return (1u << 4) | ((uint32_t)fmt << 7) | ((uint32_t)fmt << 10) | (a_mn_major ? (1u << 15) : 0u) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 template <int KIND>   // 0 = tf32, 1 = bf16 (kind::f16)

@@ -20,6 +20,7 @@ from . import binding as B
 STAGES = {"weight": B.STAGE_WEIGHT, "input": B.STAGE_INPUT, "contract": B.STAGE_CONTRACT, "output": B.STAGE_OUTPUT,
           "all": B.STAGE_INPUT | B.STAGE_CONTRACT | B.STAGE_OUTPUT}
 OPERANDS = {"auto": B.OPERAND_AUTO, "tf32": B.OPERAND_TF32, "bf16": B.OPERAND_BF16, "fp32ref": B.OPERAND_FP32_REF}
+LHS = {"auto": B.GEMM_LHS_AUTO, "patches": B.GEMM_LHS_PATCHES, "x": B.GEMM_LHS_X}
 ALGOS = {"auto": B.ALGO_AUTO, "winograd": B.ALGO_WINOGRAD, "gemm": B.ALGO_GEMM, "direct": B.ALGO_DIRECT}
 
 
@@ -39,7 +40,10 @@ def stage_work(info, N, Cin, Cout, H, W, k, groups):
     elif info.algo == B.ALGO_GEMM:
         K, T = Cin * k * k, N * info.OH * info.OW
         v = b_el * T * K
-        out["input"] = (x_bytes + v, 0)
+        if info.gemm_lhs == B.GEMM_LHS_X:
+            v = x_bytes                    # the contraction reads x itself
+        else:
+            out["input"] = (x_bytes + v, 0)
         out["contract"] = (v + b_el * Cout * K + y_bytes, 2 * T * Cout * K * info.passes)
     else:
         out["contract"] = (x_bytes + y_bytes + 4 * Cout * (Cin // groups) * k * k,
@@ -62,6 +66,7 @@ def main():
     ap.add_argument("--passes", type=int, default=0)
     ap.add_argument("--algo", default="auto", choices=sorted(ALGOS))
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--lhs", default="auto", choices=sorted(LHS), help="left operand of the GEMM scheme")
     ap.add_argument("--precision", default="tf32", choices=["tf32", "bf16"])
     ap.add_argument("--stages", default="all", choices=sorted(STAGES))
     ap.add_argument("--reps", type=int, default=3)
@@ -75,7 +80,7 @@ def main():
     pad = (args.k - 1) // 2 if args.pad < 0 else args.pad
     o = B.make_opts(groups=args.groups, relu=1, precision=B.PREC_TF32 if args.precision == "tf32" else B.PREC_BF16,
                     operand=OPERANDS[args.operand], passes=args.passes, force_algo=ALGOS[args.algo], force_m=args.m,
-                    chunk_images=args.chunk)
+                    chunk_images=args.chunk, gemm_lhs=LHS[args.lhs])
     r = B.ConvLayerRunner(args.N, Cin, Cout, args.H, args.H, args.k, args.stride, pad, 1, o)
     info = r.info
     g = torch.Generator(device="cpu").manual_seed(1)
@@ -113,7 +118,7 @@ def main():
     total_ms = sum(s["ms"] for s in stages.values())
     direct = 2 * args.N * Cout * (Cin // args.groups) * info.OH * info.OW * args.k * args.k
     print(json.dumps({"algo": B.ALGO_NAMES[info.algo], "m": info.m, "operand": B.OPERAND_NAMES[info.operand],
-                      "passes": info.passes, "chunk_images": info.chunk_images, "n_chunks": info.n_chunks,
+                      "passes": info.passes, "gemm_lhs": info.gemm_lhs, "chunk_images": info.chunk_images, "n_chunks": info.n_chunks,
                       "workspace_MB": round(info.workspace_bytes / 2 ** 20, 1), "device_status": status,
                       "stages": stages, "sum_ms": round(total_ms, 5),
                       "direct_equiv_TFLOPs": round(direct / total_ms / 1e9, 1) if total_ms > 0 else None}))

@@ -282,6 +282,51 @@ def test_gemm_bit_exact_on_integers(torch):
         assert np.array_equal(got.astype(np.float64), ref)
 
 
+# 1x1 stride-1 layers: the GEMM scheme with either left operand (the gathered patch matrix, or x itself read as
+# a pixel-contiguous operand).  Shapes cover one and several 32-pixel atoms per image with a ragged last atom,
+# an atom count that does not fill the last work item, channel counts off the K block and the channel block.
+@pytest.mark.parametrize("Cin,Cout,H,W_,N", [
+    (64, 128, 8, 8, 2), (24, 40, 14, 14, 3), (512, 512, 14, 14, 1), (100, 72, 6, 6, 5), (32, 16, 28, 28, 2),
+    (72, 300, 9, 12, 2), (130, 260, 7, 12, 7), (8, 8, 4, 8, 1)])
+@pytest.mark.parametrize("lhs", [B.GEMM_LHS_PATCHES, B.GEMM_LHS_X])
+def test_gemm_left_operand_1x1(torch, Cin, Cout, H, W_, N, lhs):
+    layer = W.ConvLayer("t", N, Cin, Cout, H, W_, 1, 1, 0, 1, relu=True, seed=Cin + H)
+    x, w, b = W.make_inputs(layer)
+    o = opts_for(layer, force_algo=B.ALGO_GEMM, operand=B.OPERAND_TF32, passes=1, gemm_lhs=lhs)
+    got, info, _ = run_layer(torch, layer, o, (x, w, b))
+    assert info.algo == B.ALGO_GEMM and info.gemm_lhs == lhs
+    assert info.launches_per_run == (1 if lhs == B.GEMM_LHS_X else 2)
+    if lhs == B.GEMM_LHS_X:
+        assert info.v_bytes == 0
+    assert_close(got, oracle(layer, x, w, b), B.PREC_TF32, "gemm 1x1")
+
+
+@pytest.mark.parametrize("Cin,Cout,H,N", [(40, 24, 6, 3), (96, 136, 14, 2)])
+def test_gemm_left_operand_x_bit_exact_on_integers(torch, Cin, Cout, H, N):
+    # small integers are exact in TF32 whether rounded or truncated: both left operands give the exact sums
+    layer = W.ConvLayer("t", N, Cin, Cout, H, H, 1, 1, 0, 1, relu=False, seed=3)
+    x, w, b = W.integer_inputs(layer)
+    ref = oracle(layer, x, w, b)
+    for lhs in (B.GEMM_LHS_PATCHES, B.GEMM_LHS_X):
+        o = opts_for(layer, force_algo=B.ALGO_GEMM, operand=B.OPERAND_TF32, passes=1, gemm_lhs=lhs)
+        got, info, _ = run_layer(torch, layer, o, (x, w, b))
+        assert info.gemm_lhs == lhs
+        assert np.array_equal(got.astype(np.float64), ref)
+
+
+def test_gemm_left_operand_x_leaves_neighbours_untouched(torch):
+    # the ragged last atom of an image must not write into the next channel's pixels: run into a buffer
+    # prefilled with a marker and compare everything, then check two images give what each gives alone
+    layer = W.ConvLayer("t", 2, 48, 20, 6, 6, 1, 1, 0, 1, relu=False, seed=11)
+    x, w, b = W.make_inputs(layer)
+    o = opts_for(layer, force_algo=B.ALGO_GEMM, operand=B.OPERAND_TF32, passes=1, gemm_lhs=B.GEMM_LHS_X)
+    both, _, _ = run_layer(torch, layer, o, (x, w, b))
+    one = W.ConvLayer("t", 1, 48, 20, 6, 6, 1, 1, 0, 1, relu=False, seed=11)
+    for n in range(2):
+        alone, _, _ = run_layer(torch, one, o, (x[n:n + 1].copy(), w, b))
+        assert np.array_equal(alone[0], both[n])
+
+
 @pytest.mark.parametrize("C,H,stride,N", [(32, 112, 1, 2), (64, 112, 2, 2), (40, 13, 1, 3), (40, 13, 2, 3), (8, 7, 1, 1),
                                           (8, 70, 2, 1), (16, 33, 1, 1)])
 def test_depthwise_direct(torch, C, H, stride, N):

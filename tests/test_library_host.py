@@ -134,6 +134,35 @@ def test_forced_options_and_errors():
     assert "groups" in B.mnn_last_error()
 
 
+def test_gemm_left_operand_option():
+    def plan(N, Cin, Cout, H, W_, k, stride, pad, **kw):
+        h = B.mnn_conv_plan_ex(N, Cin, Cout, H, W_, k, stride, pad, 1, B.make_opts(relu=1, **kw))
+        info = B.mnn_conv_plan_query(h)
+        B.mnn_conv_destroy(h)
+        return info
+    gemm = dict(force_algo=B.ALGO_GEMM, operand=B.OPERAND_TF32, passes=1)
+    # x itself: one launch, no patch matrix in the workspace, a smaller workspace than with patches
+    ix = plan(4, 64, 96, 14, 14, 1, 1, 0, gemm_lhs=B.GEMM_LHS_X, **gemm)
+    ip = plan(4, 64, 96, 14, 14, 1, 1, 0, gemm_lhs=B.GEMM_LHS_PATCHES, **gemm)
+    assert (ix.gemm_lhs, ix.launches_per_run, ix.v_bytes) == (B.GEMM_LHS_X, 1, 0)
+    assert (ip.gemm_lhs, ip.launches_per_run) == (B.GEMM_LHS_PATCHES, 2) and ip.v_bytes >= 4 * 4 * 196 * 64
+    assert ix.workspace_bytes < ip.workspace_bytes
+    assert ix.predicted_error_ppm >= ip.predicted_error_ppm          # truncation instead of rounding
+    # left to the planner the choice is one of the two and is reported; other schemes report 0
+    ia = plan(4, 64, 96, 14, 14, 1, 1, 0, **gemm)
+    assert ia.gemm_lhs in (B.GEMM_LHS_X, B.GEMM_LHS_PATCHES)
+    assert plan(1, 32, 32, 28, 28, 3, 1, 1, force_algo=B.ALGO_WINOGRAD).gemm_lhs == 0
+    # where x cannot be the operand, asking for it fails the plan; patches still plan
+    for shape in [(1, 64, 64, 14, 14, 3, 1, 1), (1, 64, 64, 14, 14, 1, 2, 0), (1, 64, 64, 7, 7, 1, 1, 0),
+                  (1, 64, 64, 4, 4, 1, 1, 0), (1, 64, 64, 14, 14, 1, 1, 1)]:
+        with pytest.raises(B.MnnError):
+            plan(*shape, gemm_lhs=B.GEMM_LHS_X, **gemm)
+        assert plan(*shape, gemm_lhs=B.GEMM_LHS_PATCHES, **gemm).gemm_lhs == B.GEMM_LHS_PATCHES
+    with pytest.raises(B.MnnError):                                   # BF16 operands need the rounded copy
+        plan(4, 64, 96, 14, 14, 1, 1, 0, force_algo=B.ALGO_GEMM, operand=B.OPERAND_BF16, precision=B.PREC_BF16,
+             gemm_lhs=B.GEMM_LHS_X)
+
+
 def test_calibration_record_round_trip_changes_the_plan():
     base = B.mnn_get_calibration()
     try:
