@@ -30,7 +30,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (mean over the four layers of one step) from one ncu
 # capture of this file's default workload (profiles/bench_config1_b32_launch_list.md gives the command).  Valid
 # for config1_b32 / tf32 and the kernels as captured; set an entry to None when its kernel changes.
-NCU_DRAM_BYTES_PER_LAUNCH = {"config1_b32/tf32": {"input": 40.38e6, "contraction": 45.51e6, "output": 15.71e6}}
+NCU_DRAM_BYTES_PER_LAUNCH = {"config1_b32/tf32": {"input": 40.36e6, "contraction": 45.23e6, "output": 15.63e6}}
 
 
 def workload_layers(name: str):
@@ -218,6 +218,9 @@ def main():
     ap.add_argument("--workload", default="config1_b32")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--precision", default="tf32", choices=["tf32", "bf16"])
+    ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
+                    help="how a timed step is issued: one CUDA-graph replay of the step's launches (captured "
+                         "once from the same C-ABI calls), or the calls themselves on the stream")
     ap.add_argument("--calibration", default="measure", choices=["measure", "builtin"],
                     help="measure: run mnn_calibrate on this GPU before planning (default); builtin: plan from the "
                          "library's frozen B200 record (use under a profiler, which slows the calibration launches)")
@@ -286,6 +289,19 @@ def main():
     for s in state:
         assert s["runner"].device_status() == 0, "a kernel reported a bounded wait that ran out"
 
+    # The step's launches captured once into a CUDA graph: the same C-ABI calls, recorded instead of run.
+    # Replaying it issues the same kernels with the same arguments without the per-launch host work.
+    timed_step = one_step
+    if args.launch == "graph":
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(step_graph):
+            one_step()
+        timed_step = step_graph.replay
+        for _ in range(3):
+            flush.zero_()
+            timed_step()
+        barrier()
+
     # ---- timed region: K steps, L2 flushed before each, device time by CUDA events ----
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -296,7 +312,7 @@ def main():
     for k in range(args.steps):
         flush.zero_()
         ev[k][0].record(stream)
-        one_step()
+        timed_step()
         ev[k][1].record(stream)
     barrier()
     t_wall1 = time.time()
@@ -419,6 +435,7 @@ def main():
                 "data": "synthetic",
                 "config": {"workload": args.workload, "layers": len(layers), "batch_per_gpu": layers[0].N,
                            "l2": "flushed before every step (256 MB write)", "weights": "pre-transformed",
+                           "launch": "CUDA graph replay per step" if args.launch == "graph" else "C-ABI calls on the stream",
                            "accuracy_class": args.precision, "planner_calibration": calibration[:9], "calibration_source": args.calibration, "plans": per_layer},
                 "clocks": clocks, "roofline": roofline,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -349,6 +349,134 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
     }
 }
 
+// The same sweep for even image widths, with VIN = 2 or 4 input columns per lane (W a multiple of VIN): rows are
+// read and written with aligned 64- or 128-bit accesses, a warp keeps four whole rows of up to 512 bytes in
+// flight, and a lane needs one value from its left neighbour per row (and one from its right neighbour at
+// stride 1).  A lane holds input columns icol0 + [0, VIN) of its plane and produces VIN outputs (stride 1) or
+// VIN / 2 (stride 2).  Planes no wider than SW * VIN take one strip with every lane productive; wider ones are
+// cut into strips that overlap by one lane on the left (and one on the right at stride 1) whose columns the
+// neighbouring strip produces.
+template <int VIN>
+struct DwRow {
+    float e[VIN + 2];      // e[0] left neighbour, e[1 .. VIN] own columns, e[VIN + 1] right neighbour (stride 1)
+};
+
+template <int VIN>
+__device__ __forceinline__ void dw_load_row(const float* __restrict__ p, bool ok, DwRow<VIN>& r)
+{
+    if (VIN == 4) {
+        const float4 v = ok ? __ldg(reinterpret_cast<const float4*>(p)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        r.e[1] = v.x; r.e[2] = v.y; r.e[3] = v.z; r.e[VIN] = v.w;
+    } else {
+        const float2 v = ok ? __ldg(reinterpret_cast<const float2*>(p)) : make_float2(0.f, 0.f);
+        r.e[1] = v.x; r.e[VIN] = v.y;
+    }
+}
+
+template <int STRIDE, int SW, int VIN>
+__global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __restrict__ x, const float* __restrict__ w,
+                                                               const float* __restrict__ bias, float* __restrict__ y,
+                                                               DirectGeom g, int strips, int bands, long long n_planes,
+                                                               long long n_units)
+{
+    constexpr int PPW = 32 / SW;                      // planes per warp
+    constexpr int VOUT = STRIDE == 1 ? VIN : VIN / 2;
+    const int lane = threadIdx.x & 31, ls = lane % SW, seg = lane / SW;
+    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (plane group, band, strip)
+    if (unit >= n_units) return;
+    const int strip = (int)(unit % strips);
+    const long long rest = unit / strips;
+    const int band = (int)(rest % bands);
+    const long long plane = (rest / bands) * PPW + seg;
+    const bool plane_ok = plane < n_planes;
+    const int c = (int)((plane_ok ? plane : 0) % g.Cout);
+    const float* xp = x + (size_t)(plane_ok ? plane : 0) * g.H * g.W;
+    float* yp = y + (size_t)(plane_ok ? plane : 0) * g.OH * g.OW;
+    float wk[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + (size_t)c * 9 + i);
+    const float b = bias ? __ldg(bias + c) : 0.0f;
+    const int oh0 = band * kDwBandRows, oh1 = min(g.OH, oh0 + kDwBandRows);
+    const unsigned full = 0xffffffffu;
+
+    // columns of this lane
+    const int lanes_per_strip = STRIDE == 1 ? SW - 2 : SW - 1;            // productive lanes of an overlapping strip
+    const int in_base = strips == 1 ? 0 : strip * lanes_per_strip * VIN - VIN;
+    const int icol0 = in_base + ls * VIN;
+    const bool col_ok = plane_ok && icol0 >= 0 && icol0 < g.W;            // the whole vector lies inside or outside
+    const bool owns = col_ok && (ls >= 1 || strips == 1) && (STRIDE == 2 || ls <= SW - 2 || strip == strips - 1);
+    const int ocol0 = STRIDE == 1 ? icol0 : icol0 / 2;
+    auto load = [&](int ih, DwRow<VIN>& r) {
+        const bool ok = col_ok && ih >= 0 && ih < g.H;
+        dw_load_row<VIN>(xp + (size_t)(ok ? ih : 0) * g.W + (ok ? icol0 : 0), ok, r);
+    };
+    auto edges = [&](DwRow<VIN>& r) {                                      // neighbours' border values
+        const float l = __shfl_up_sync(full, r.e[VIN], 1, SW);
+        r.e[0] = ls == 0 ? 0.0f : l;
+        if (STRIDE == 1) {
+            const float q = __shfl_down_sync(full, r.e[1], 1, SW);
+            r.e[VIN + 1] = ls == SW - 1 ? 0.0f : q;
+        }
+    };
+    auto out = [&](int oh, const DwRow<VIN>& a, const DwRow<VIN>& m, const DwRow<VIN>& z) {
+        float acc[VOUT];
+#pragma unroll
+        for (int j = 0; j < VOUT; ++j) {
+            float v = b;
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                v = fmaf(wk[t], a.e[STRIDE * j + t], v);
+                v = fmaf(wk[3 + t], m.e[STRIDE * j + t], v);
+                v = fmaf(wk[6 + t], z.e[STRIDE * j + t], v);
+            }
+            acc[j] = g.relu ? fmaxf(v, 0.0f) : v;
+        }
+        if (owns) {
+            float* q = yp + (size_t)oh * g.OW + ocol0;
+            if (VOUT == 4) *reinterpret_cast<float4*>(q) = make_float4(acc[0], acc[1], acc[2], acc[VOUT - 1]);
+            else if (VOUT == 2) *reinterpret_cast<float2*>(q) = make_float2(acc[0], acc[VOUT - 1]);
+            else *q = acc[0];
+        }
+    };
+
+    if (STRIDE == 1) {
+        DwRow<VIN> r0, r1;
+        load(oh0 - 1, r0);
+        load(oh0, r1);
+        edges(r0);
+        edges(r1);
+        for (int oh = oh0; oh < oh1; oh += 4) {
+            DwRow<VIN> nx[4];                         // input rows oh + 1 .. oh + 4, all requested before use
+#pragma unroll
+            for (int k = 0; k < 4; ++k) load(oh + k + 1, nx[k]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (oh + k < oh1) {
+                    edges(nx[k]);
+                    out(oh + k, r0, r1, nx[k]);
+                    r0 = r1;
+                    r1 = nx[k];
+                }
+            }
+        }
+    } else {
+        DwRow<VIN> prev;
+        load(2 * oh0 - 1, prev);
+        edges(prev);
+        for (int oh = oh0; oh < oh1; oh += 2) {
+            DwRow<VIN> ra, rb, rc, rd;                // input rows 2 oh .. 2 oh + 3, all requested before use
+            load(2 * oh, ra);
+            load(2 * oh + 1, rb);
+            load(2 * oh + 2, rc);
+            load(2 * oh + 3, rd);
+            edges(ra); edges(rb); edges(rc); edges(rd);
+            out(oh, prev, ra, rb);
+            if (oh + 1 < oh1) out(oh + 1, rb, rc, rd);
+            prev = rd;
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_gather(const float* x, void* V_hi, void* V_lo, const GatherGeom& g, int mode, cudaStream_t stream)
@@ -387,12 +515,34 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
                             (g.stride == 1 || g.stride == 2);
     if (depthwise3) {
         const long long planes = (long long)g.N * g.Cout;
-        // lanes per plane segment: a stride-1 segment of SW lanes covers SW - 1 input columns from -1 on, a
-        // stride-2 segment SW output columns
+        const int bands = (g.OH + kDwBandRows - 1) / kDwBandRows;
+        if (g.W % 2 == 0) {
+            // even widths: 2 or 4 columns per lane, the narrowest segment that holds a row, else 32-lane strips
+            const int vin = g.W % 4 == 0 ? 4 : 2;
+            const int need = g.W / vin;
+            const int sw = need <= 8 ? 8 : (need <= 16 ? 16 : 32);
+            const int per_strip = (g.stride == 1 ? 30 : 31) * vin;
+            const int strips = need <= 32 ? 1 : (g.W + per_strip - 1) / per_strip;
+            const long long groups = (planes + 32 / sw - 1) / (32 / sw);
+            const long long units = groups * strips * bands;
+            const long long blocks = (units + 3) / 4;
+            if (blocks > 2147483647ll) return cudaErrorInvalidValue;
+#define MNNB_DWV_LAUNCH(ST, SWV, VI) depthwise3x3_vec_kernel<ST, SWV, VI><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, planes, units)
+#define MNNB_DWV_PICK(ST, VI) do { if (sw == 8) MNNB_DWV_LAUNCH(ST, 8, VI); else if (sw == 16) MNNB_DWV_LAUNCH(ST, 16, VI); else MNNB_DWV_LAUNCH(ST, 32, VI); } while (0)
+            if (g.stride == 1) {
+                if (vin == 4) MNNB_DWV_PICK(1, 4); else MNNB_DWV_PICK(1, 2);
+            } else {
+                if (vin == 4) MNNB_DWV_PICK(2, 4); else MNNB_DWV_PICK(2, 2);
+            }
+#undef MNNB_DWV_PICK
+#undef MNNB_DWV_LAUNCH
+            return cudaGetLastError();
+        }
+        // odd widths: one column per lane.  A stride-1 segment of SW lanes covers SW - 1 input columns from -1
+        // on, a stride-2 segment SW output columns
         const int need = g.stride == 1 ? g.W + 1 : g.OW;
         const int sw = need <= 8 ? 8 : (need <= 16 ? 16 : 32);
         const int strips = sw < 32 ? 1 : (g.stride == 1 ? (g.OW + 29) / 30 : (g.OW + 31) / 32);
-        const int bands = (g.OH + kDwBandRows - 1) / kDwBandRows;
         const long long groups = (planes + 32 / sw - 1) / (32 / sw);
         const long long units = groups * strips * bands;
         const long long blocks = (units + 3) / 4;

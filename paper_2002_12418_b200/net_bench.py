@@ -20,6 +20,9 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--reps", type=int, default=50)
+    ap.add_argument("--calibration", default="measure", choices=["measure", "builtin"],
+                    help="builtin plans from the library's frozen record (use it under a profiler, which slows "
+                         "the calibration's own launches)")
     args = ap.parse_args()
     import torch
     B.lib()
@@ -27,7 +30,8 @@ def main():
     torch.cuda.set_device(dev)
     N = args.batch
     layers = W.config3(N)
-    B.mnn_calibrate(0, torch.cuda.current_stream().cuda_stream)
+    if args.calibration == "measure":
+        B.mnn_calibrate(0, torch.cuda.current_stream().cuda_stream)
     x = torch.from_numpy(W.make_inputs(layers[0])[0]).to(dev)
     ws, bs = [], []
     for l in layers:

@@ -337,6 +337,27 @@ def test_depthwise_direct(torch, C, H, stride, N):
     assert rel_l2(got, oracle(layer, x, w, b)) < 1e-6
 
 
+# Even widths take the depthwise kernel with 2 or 4 columns per lane: widths that fill 8, 16 and 32 lanes, that
+# need two and three overlapping strips, heights off the 32-row band and odd, plane counts that leave a warp
+# partly empty, both strides.
+@pytest.mark.parametrize("C,H,W_,N", [(10, 14, 14, 3), (7, 28, 28, 2), (6, 56, 56, 1), (3, 112, 112, 1), (2, 40, 224, 1),
+                                      (3, 9, 130, 2), (5, 15, 6, 1), (4, 67, 36, 1), (1, 33, 248, 1), (9, 5, 2, 1),
+                                      (2, 3, 500, 1)])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_depthwise_even_widths(torch, C, H, W_, N, stride):
+    layer = W.ConvLayer("t", N, C, C, H, W_, 3, stride, 1, groups=C, relu=(C % 2 == 0), seed=C + H + W_)
+    x, w, b = W.make_inputs(layer)
+    got, info, _ = run_layer(torch, layer, opts_for(layer), (x, w, b))
+    assert info.algo == B.ALGO_DIRECT
+    ref = oracle(layer, x, w, b)
+    assert got.shape == ref.shape
+    assert rel_l2(got, ref) < 1e-6
+    # integer inputs: bit-exact, which also shows every output element was written exactly once with its own value
+    xi, wi, bi = W.integer_inputs(layer)
+    goti, _, _ = run_layer(torch, layer, opts_for(layer), (xi, wi, bi))
+    assert np.array_equal(goti.astype(np.float64), oracle(layer, xi, wi, bi))
+
+
 @pytest.mark.parametrize("Cin,Cout,H,k,stride,pad,dil,groups", [
     (3, 32, 32, 3, 2, 1, 1, 1), (3, 16, 30, 7, 2, 3, 1, 1), (6, 6, 9, 3, 1, 1, 2, 6), (5, 7, 8, 2, 1, 0, 1, 1),
     (4, 4, 6, 5, 3, 2, 1, 4)])
