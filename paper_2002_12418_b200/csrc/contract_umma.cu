@@ -19,10 +19,15 @@
 // short K loops, where the epilogue decides.)
 //
 // A 1x1 stride-1 convolution needs no patch matrix: x[n] = [Cin][H*W] already is operand A, stored with the
-// M index (the pixel) contiguous.  In that mode (a_mn) the producer copies boxes of 32 pixels x 32 channels
-// straight out of x, the MMA reads A as an MN-major operand, and a work item covers four such 32-pixel
-// "atoms" (each inside one image), one per epilogue warp.  The tensor core drops the low 13 mantissa bits of
-// the fp32 values it is given (truncation, where the stored operands are rounded to nearest).
+// M index (the pixel) contiguous.  In that mode (a_mn) the MMA reads A as an MN-major operand made of
+// "atoms" of 32 pixels x 32 channels, and a work item covers up to four consecutive atoms of ONE image, one
+// per epilogue warp.  The producer fetches the item's full atoms with a single 4-D box {32 pixels, 32
+// channels, n atoms} (x viewed as [image][atom][channel][32 pixels]; one box of 16 KB moves several times
+// faster than four boxes of 4 KB) and a ragged last atom of the image with a 3-D box over [image][channel]
+// [pixel], whose pixels past H*W read as zeros, so no read leaves x.  Atom slots of the last item of an
+// image that hold no atom are not loaded; their accumulator rows are not stored.  The tensor core drops the
+// low 13 mantissa bits of the fp32 values it is given (truncation, where the stored operands are rounded
+// to nearest).
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -48,9 +53,9 @@ struct KernelParams {
     long long n_items;
     ContractEpilogue epi;
     int* status;
-    // a_mn mode: operand A comes from x [images][Cin][hw]; 32-pixel atoms, atoms_per_image = ceil(hw / 32)
-    int a_mn, hw, atoms_per_image;
-    long long total_atoms;
+    // a_mn mode: operand A comes from x [images][Cin][hw]; atoms of 32 pixels: full_atoms = hw / 32 whole ones
+    // and a ragged one when hw % 32 != 0; tiles_per_image work items of up to four atoms cover an image
+    int a_mn, hw, full_atoms, atoms_per_image, tiles_per_image;
 };
 
 // status codes written on a bounded wait that ran out
@@ -60,7 +65,9 @@ template <int KIND>
 __global__ void __launch_bounds__(kThreads, 1)
 contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_constant__ CUtensorMap map_v_lo,
                      const __grid_constant__ CUtensorMap map_u_hi, const __grid_constant__ CUtensorMap map_u_lo,
-                     KernelParams p)
+                     const __grid_constant__ CUtensorMap map_x_ragged, KernelParams p)
+// a_mn mode: map_v_hi = 4-D map over x with the box height of an image's leading items, map_v_lo = the same with
+// the box height of its last item, map_x_ragged = 3-D map for the ragged atom.
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
@@ -131,18 +138,22 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     }
                     const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
                     const uint32_t sbase = smem_base + stage * stage_bytes;
-                    ptx::mbar_expect_tx(bar, stage_bytes);
                     if (p.a_mn) {
-#pragma unroll
-                        for (int j = 0; j < kTileM / 32; ++j) {
-                            // an atom past the end names an image that does not exist and reads as zeros
-                            const long long a = (long long)tb * (kTileM / 32) + j;
-                            const int img = (int)(a / p.atoms_per_image);
-                            const int pix0 = (int)(a - (long long)img * p.atoms_per_image) * 32;
-                            ptx::tma_load_3d(sbase + j * 4096, &map_v_hi, bar, pix0, kb * k_elems, img);
-                        }
-                    } else
+                        const int img = tb / p.tiles_per_image;
+                        const int a0 = (tb - img * p.tiles_per_image) * (kTileM / 32);       // first atom of the item
+                        const int n_full = min(kTileM / 32, max(0, p.full_atoms - a0));
+                        const bool ragged = p.full_atoms < p.atoms_per_image && a0 + kTileM / 32 >= p.atoms_per_image;
+                        ptx::mbar_expect_tx(bar, (uint32_t)(n_full + (ragged ? 1 : 0)) * 4096u + b_bytes);
+                        if (n_full > 0)
+                            ptx::tma_load_4d(sbase, a0 + kTileM / 32 <= p.full_atoms ? &map_v_hi : &map_v_lo, bar, 0,
+                                             kb * k_elems, a0, img);
+                        if (ragged)
+                            ptx::tma_load_3d(sbase + (uint32_t)n_full * 4096u, &map_x_ragged, bar, p.full_atoms * 32,
+                                             kb * k_elems, img);
+                    } else {
+                        ptx::mbar_expect_tx(bar, stage_bytes);
                         ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
+                    }
                     ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
                     if (split == 2) {
                         ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM, xi);
@@ -239,10 +250,9 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 step = p.epi.m_row_stride;
                 dst = p.epi.M + ((size_t)xi * p.Cout + co0) * p.epi.m_row_stride + t;
             } else if (p.a_mn) {
-                const long long a = (long long)tb * (kTileM / 32) + q;       // this warp's atom
-                const long long img = a / p.atoms_per_image;
-                const int pix = (int)(a - img * p.atoms_per_image) * 32 + lane;
-                t_ok = a < p.total_atoms && pix < p.hw;
+                const int img = tb / p.tiles_per_image;
+                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) + q) * 32 + lane;   // this warp's atom
+                t_ok = pix < p.hw;
                 step = p.hw;
                 dst = p.epi.y + ((size_t)(t_ok ? img : 0) * p.Cout + co0) * p.hw + (t_ok ? pix : 0);
             } else {
@@ -492,8 +502,9 @@ cudaError_t umma_contract_setup_x(UmmaContract* uc, int Cout, int Cin, int cin_p
         *why = "reading x as operand A needs H*W >= 32 and a multiple of 4";
         return cudaErrorInvalidValue;
     }
-    const long long atoms = (long long)images * ((hw + 31) / 32);
-    cudaError_t e = umma_contract_setup(uc, STORE_TF32, 1, Cout, cin_pad, atoms * 32, U, nullptr, nullptr, nullptr, why);
+    const int atoms = (hw + 31) / 32, tiles_per_image = (atoms + kTileM / 32 - 1) / (kTileM / 32);
+    cudaError_t e = umma_contract_setup(uc, STORE_TF32, 1, Cout, cin_pad, (long long)images * tiles_per_image * kTileM, U,
+                                        nullptr, nullptr, nullptr, why);
     if (e != cudaSuccess) return e;
     uc->x_images = images;
     uc->x_cin = Cin;
@@ -508,23 +519,43 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     if (!uc.ready || !uc.a_mn) return cudaErrorInvalidValue;
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return cudaErrorInvalidValue;
-    // x as [images][Cin][hw], box = 32 pixels x 32 channels of one image, 128-byte swizzle with a 32-byte base
-    CUtensorMap map_x;
-    const cuuint64_t dims[3] = {(cuuint64_t)uc.x_hw, (cuuint64_t)uc.x_cin, (cuuint64_t)uc.x_images};
-    const cuuint64_t strides[2] = {(cuuint64_t)uc.x_hw * 4, (cuuint64_t)uc.x_cin * uc.x_hw * 4};
-    const cuuint32_t box[3] = {32, 32, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    if (fn(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(x), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
     KernelParams p;
     p.a_mn = 1;
     p.hw = uc.x_hw;
+    p.full_atoms = uc.x_hw / 32;
     p.atoms_per_image = (uc.x_hw + 31) / 32;
-    p.total_atoms = (long long)uc.x_images * p.atoms_per_image;
+    p.tiles_per_image = (p.atoms_per_image + kTileM / 32 - 1) / (kTileM / 32);
+    // Tensor maps over x, 128-byte swizzle with a 32-byte base.  Whole atoms: x as [image][atom][channel][32
+    // pixels] (the atom stride, 128 bytes, is smaller than the channel stride), box = 32 pixels x 32 channels x
+    // h atoms, h = 4 for the leading items of an image and what is left for its last item.  Ragged atom: x as
+    // [image][channel][pixel], box = 32 pixels x 32 channels, pixels past hw read as zeros.
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const cuuint64_t plane = (cuuint64_t)uc.x_hw * 4;
+    auto encode_atoms = [&](CUtensorMap* m, int h) {
+        const cuuint64_t dims[4] = {32, (cuuint64_t)uc.x_cin, (cuuint64_t)p.full_atoms, (cuuint64_t)uc.x_images};
+        const cuuint64_t strides[3] = {plane, 128, (cuuint64_t)uc.x_cin * plane};
+        const cuuint32_t box[4] = {32, 32, (cuuint32_t)h, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    CUtensorMap map_lead, map_last, map_ragged;
+    const int h_lead = p.full_atoms < kTileM / 32 ? p.full_atoms : kTileM / 32;
+    int h_last = p.full_atoms - (p.tiles_per_image - 1) * (kTileM / 32);       // whole atoms of an image's last item
+    if (h_last < 1 || h_last > kTileM / 32) h_last = h_lead;                   // (none: the map is not used)
+    if (!encode_atoms(&map_lead, h_lead) || !encode_atoms(&map_last, h_last)) return cudaErrorInvalidValue;
+    {
+        const cuuint64_t dims[3] = {(cuuint64_t)uc.x_hw, (cuuint64_t)uc.x_cin, (cuuint64_t)uc.x_images};
+        const cuuint64_t strides[2] = {plane, (cuuint64_t)uc.x_cin * plane};
+        const cuuint32_t box[3] = {32, 32, 1};
+        if (fn(&map_ragged, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    if ((long long)uc.x_images * p.tiles_per_image > 2147483647ll) return cudaErrorInvalidValue;
     p.alpha2 = 1;
-    p.n_tile_blocks = (int)((p.total_atoms + kTileM / 32 - 1) / (kTileM / 32));
+    p.n_tile_blocks = uc.x_images * p.tiles_per_image;
     p.n_co_blocks = uc.n_co_blocks;
     p.bn = uc.bn;
     p.k_blocks = uc.k_blocks;
@@ -532,13 +563,13 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.stages = uc.stages;
     p.tmem_cols = uc.tmem_cols;
     p.Cout = uc.Cout;
-    p.tiles = p.total_atoms * 32;
+    p.tiles = (long long)p.n_tile_blocks * kTileM;
     p.n_items = (long long)p.n_tile_blocks * p.n_co_blocks;
     p.epi = epi;
     p.status = status;
     const long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
     return launch_overlapped(contract_umma_kernel<0>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
-                             map_x, map_x, uc.map_u_hi, uc.map_u_lo, p);
+                             map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
 }
 
 cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const ContractEpilogue& epi, int* status,
@@ -550,8 +581,9 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     KernelParams p;
     p.a_mn = 0;
     p.hw = 0;
+    p.full_atoms = 0;
     p.atoms_per_image = 1;
-    p.total_atoms = 0;
+    p.tiles_per_image = 1;
     p.alpha2 = uc.alpha2;
     p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
     p.n_co_blocks = uc.n_co_blocks;
@@ -568,9 +600,9 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
     if (uc.kind == 0)
         return launch_overlapped(contract_umma_kernel<0>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
-                                 uc.map_v_hi, uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, p);
+                                 uc.map_v_hi, uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
     return launch_overlapped(contract_umma_kernel<1>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
-                             uc.map_v_hi, uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, p);
+                             uc.map_v_hi, uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
 }
 
 }  // namespace mnnb

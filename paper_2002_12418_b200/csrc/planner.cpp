@@ -348,14 +348,16 @@ uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibrati
     const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3 : 10) / 2, 0, 0, cal);
     // The contraction as the kernel schedules it: rounds of work items over the SMs, each item a serial loop
     // over blocks of K whose pace is the slower of the tensor core and the delivery of the two operand tiles
-    // from L2 to one SM (about 63 GB/s measured; about 21 GB/s for the pixel-contiguous tile read out of x).
+    // from L2 to one SM (about 63 GB/s measured, for either left operand).  With x as the left operand a work
+    // item covers up to four 32-pixel atoms of one image, so images whose atom count is not a multiple of four
+    // leave part of their last item empty.
     const int sms = cal.c[7] > 0 ? (int)cal.c[7] : 148;
-    const uint64_t tile_blocks = lhs_x ? ceil_div((uint64_t)s.N * ceil_div((uint64_t)s.H * s.W, 32), 4) : ceil_div(T, 128);
+    const uint64_t tile_blocks = lhs_x ? (uint64_t)s.N * ceil_div(ceil_div((uint64_t)s.H * s.W, 32), 4) : ceil_div(T, 128);
     int bn = 256, n_co_blocks = 1;
     contract_tiling((long long)tile_blocks, 1, s.Cout, sms, &bn, &n_co_blocks);
     const uint64_t rounds = ceil_div(tile_blocks * (uint64_t)n_co_blocks, (uint64_t)sms);
     const uint64_t k_elems = 128 / b, k_blocks = ceil_div(Kp, k_elems);
-    const uint64_t deliver_ps = 128ull * 128 * (lhs_x ? 46 : 16) + (uint64_t)bn * 128 * 16;
+    const uint64_t deliver_ps = (128ull * 128 + (uint64_t)bn * 128) * 16;
     const uint64_t mma_ps = 2ull * 128 * bn * k_elems * tensor_as(operand, cal) * sms / 1000000ull;
     const uint64_t serial_as = rounds * k_blocks * (deliver_ps > mma_ps ? deliver_ps : mma_ps) * 1000000ull;
     if (lhs_x) return kernel_ps((x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);

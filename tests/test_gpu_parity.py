@@ -284,10 +284,12 @@ def test_gemm_bit_exact_on_integers(torch):
 
 # 1x1 stride-1 layers: the GEMM scheme with either left operand (the gathered patch matrix, or x itself read as
 # a pixel-contiguous operand).  Shapes cover one and several 32-pixel atoms per image with a ragged last atom,
-# an atom count that does not fill the last work item, channel counts off the K block and the channel block.
+# an atom count that does not fill the last work item, exactly four atoms, a last item of whole atoms only, a
+# last item holding only the ragged atom, channel counts off the K block and the channel block.
 @pytest.mark.parametrize("Cin,Cout,H,W_,N", [
     (64, 128, 8, 8, 2), (24, 40, 14, 14, 3), (512, 512, 14, 14, 1), (100, 72, 6, 6, 5), (32, 16, 28, 28, 2),
-    (72, 300, 9, 12, 2), (130, 260, 7, 12, 7), (8, 8, 4, 8, 1)])
+    (72, 300, 9, 12, 2), (130, 260, 7, 12, 7), (8, 8, 4, 8, 1), (16, 24, 8, 16, 2), (40, 48, 10, 16, 2),
+    (33, 20, 16, 18, 1), (20, 24, 4, 9, 3)])
 @pytest.mark.parametrize("lhs", [B.GEMM_LHS_PATCHES, B.GEMM_LHS_X])
 def test_gemm_left_operand_1x1(torch, Cin, Cout, H, W_, N, lhs):
     layer = W.ConvLayer("t", N, Cin, Cout, H, W_, 1, 1, 0, 1, relu=True, seed=Cin + H)
