@@ -191,11 +191,12 @@ extern "C" int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CO
         cal.c[8] = to_ll(t * 1e15 / flops);
     }
 
-    // rate of the direct kernel for very few input channels: 3x3 stride 2, 3 -> 32 channels, 224 x 224, 4 images
+    // rate of the direct kernel for very few input channels: 3x3 stride 2, 3 -> 32 channels, 224 x 224, 32 images
+    // (several waves of CTAs: a handful of images would measure the ramp-up instead of the rate)
     {
-        DirectGeom g = {4, 3, 32, 224, 224, 112, 112, 3, 2, 1, 1, 1, 1};
+        DirectGeom g = {32, 3, 32, 224, 224, 112, 112, 3, 2, 1, 1, 1, 1};
         float* x = reinterpret_cast<float*>(buf);
-        float* w = x + (size_t)4 * 3 * 224 * 224;
+        float* w = x + (size_t)32 * 3 * 224 * 224;
         float* y = w + 32 * 27 + 32;
         if (direct_stem_applies(g)) {
             for (int i = 0; i < 2; ++i) launch_direct(x, w, nullptr, y, g, st);
@@ -203,7 +204,7 @@ extern "C" int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CO
             const int reps = 5;
             for (int i = 0; i < reps; ++i) launch_direct(x, w, nullptr, y, g, st);
             ms = tm.stop();
-            const double flops = 2.0 * 4 * 32 * 3 * 112 * 112 * 9;
+            const double flops = 2.0 * 32 * 32 * 3 * 112 * 112 * 9;
             double t = ms / reps - launch_ms;
             if (t < ms / reps * 0.25) t = ms / reps * 0.25;
             cal.c[9] = to_ll(t * 1e15 / flops);

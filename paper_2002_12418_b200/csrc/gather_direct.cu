@@ -42,6 +42,38 @@ __device__ __forceinline__ void store_operand_g(void* hi, void* lo, size_t idx, 
     }
 }
 
+// Four consecutive elements of a row of V (idx a multiple of 4) in the operand format of MODE.
+template <int MODE>
+__device__ __forceinline__ void store_quad_g(void* V_hi, void* V_lo, size_t idx, const float (&v)[4])
+{
+    if (MODE == STORE_BF16 || MODE == STORE_BF16_SPLIT) {
+        __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&h01);
+        pk.y = *reinterpret_cast<uint32_t*>(&h23);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(V_hi) + idx) = pk;
+        if (MODE == STORE_BF16_SPLIT) {
+            const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+            __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y),
+                           l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+            pk.x = *reinterpret_cast<uint32_t*>(&l01);
+            pk.y = *reinterpret_cast<uint32_t*>(&l23);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(V_lo) + idx) = pk;
+        }
+    } else if (MODE == STORE_FP32) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_hi) + idx) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+        float h[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) h[e] = round_tf32_g(v[e]);
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_hi) + idx) = make_float4(h[0], h[1], h[2], h[3]);
+        if (MODE == STORE_TF32_SPLIT)
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_lo) + idx) =
+                make_float4(round_tf32_g(v[0] - h[0]), round_tf32_g(v[1] - h[1]), round_tf32_g(v[2] - h[2]),
+                            round_tf32_g(v[3] - h[3]));
+    }
+}
+
 // Generic gather: a 32 x 32 (output position x patch element) block per CTA is read
 // with the output position fastest (adjacent pixels of x), transposed through
 // shared memory and written with the patch element fastest (rows of V).
@@ -118,33 +150,131 @@ __global__ void __launch_bounds__(256) gather_1x1_kernel(const float* __restrict
         float v[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) v[e] = tile[cv + e][p];
-        if (MODE == STORE_BF16 || MODE == STORE_BF16_SPLIT) {
-            __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
-            uint2 pk;
-            pk.x = *reinterpret_cast<uint32_t*>(&h01);
-            pk.y = *reinterpret_cast<uint32_t*>(&h23);
-            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(V_hi) + idx) = pk;
-            if (MODE == STORE_BF16_SPLIT) {
-                const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-                __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y),
-                               l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
-                pk.x = *reinterpret_cast<uint32_t*>(&l01);
-                pk.y = *reinterpret_cast<uint32_t*>(&l23);
-                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(V_lo) + idx) = pk;
-            }
-        } else if (MODE == STORE_FP32) {
-            *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_hi) + idx) = make_float4(v[0], v[1], v[2], v[3]);
-        } else {
-            float h[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) h[e] = round_tf32_g(v[e]);
-            *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_hi) + idx) = make_float4(h[0], h[1], h[2], h[3]);
-            if (MODE == STORE_TF32_SPLIT)
-                *reinterpret_cast<float4*>(reinterpret_cast<float*>(V_lo) + idx) =
-                    make_float4(round_tf32_g(v[0] - h[0]), round_tf32_g(v[1] - h[1]), round_tf32_g(v[2] - h[2]),
-                                round_tf32_g(v[3] - h[3]));
+        store_quad_g<MODE>(V_hi, V_lo, idx, v);
+    }
+}
+
+// Staged gather for k > 1 layers.  A CTA owns a block of output positions of one image (rt rows x
+// seg_w columns) and a slab of patch elements (slab_q groups of four, i.e. whole 16-byte
+// pieces of the rows of V; 64 positions, or up to 256 where the rows of V are short).  It copies the input region those positions touch, for the channels of the slab,
+// into shared memory row by row (coalesced, zero outside the image), builds two offset tables (patch element
+// -> offset inside the region, position -> offset of its window's corner) and then writes V: eight lanes
+// cover 128 contiguous bytes of one row of V, a warp four rows at a time.  An element is region[koff + poff]:
+// no division or bounds test per element.
+struct StagedGather {
+    int seg_w, segs, rt, row_tiles, rh, rw, slab_q, kq_n;
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(256) gather_staged_kernel(const float* __restrict__ x, void* V_hi, void* V_lo, GatherGeom g,
+                                                            StagedGather sg)
+{
+    extern __shared__ __align__(16) unsigned char gs_raw[];
+    int* koff = reinterpret_cast<int*>(gs_raw);                 // [slab_q * 4], -1 = padding element
+    int* poff = koff + sg.slab_q * 4;                           // [256], -1 = no such position
+    float* region = reinterpret_cast<float*>(poff + 256);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k2 = g.k * g.k, Kd = g.Cin * k2;
+    const int kq0 = blockIdx.y * sg.slab_q, kq1 = min(sg.kq_n, kq0 + sg.slab_q);
+    const int kk0 = 4 * kq0, kk1 = min(4 * kq1, Kd);            // real patch elements of the slab
+    const int ci_lo = kk0 / k2, ci_hi = kk1 > kk0 ? (kk1 - 1) / k2 : ci_lo - 1;
+    int bx = blockIdx.x;
+    const int seg = bx % sg.segs; bx /= sg.segs;
+    const int rtile = bx % sg.row_tiles;
+    const int n = bx / sg.row_tiles;
+    const int oh0 = rtile * sg.rt, rows = min(sg.rt, g.OH - oh0);
+    const int ow0 = seg * sg.seg_w, cols = min(sg.seg_w, g.OW - ow0);
+    const int ih0 = oh0 * g.stride - g.pad, iw0 = ow0 * g.stride - g.pad;
+    const int plane = sg.rh * sg.rw;
+
+    for (int i = threadIdx.x; i < (kq1 - kq0) * 4; i += 256) {
+        const int kk = kk0 + i;
+        int o = -1;
+        if (kk < Kd) {
+            const int ci = kk / k2, e = kk - ci * k2, a = e / g.k, b = e - a * g.k;
+            o = (ci - ci_lo) * plane + a * g.dil * sg.rw + b * g.dil;
+        }
+        koff[i] = o;
+    }
+    {
+        const int r = threadIdx.x / sg.seg_w, c = threadIdx.x - r * sg.seg_w;
+        poff[threadIdx.x] = (r < rows && c < cols) ? r * g.stride * sg.rw + c * g.stride : -1;
+    }
+    // region rows: a warp takes 32 / lw rows per pass, lw = the power of two that covers a row (at most 32)
+    const int n_rows = (ci_hi - ci_lo + 1) * sg.rh;
+    int lw = 32;
+    while (lw > 1 && (lw >> 1) >= sg.rw) lw >>= 1;
+    const int rows_per_pass = 32 / lw, sub = lane / lw, lc = lane - sub * lw;
+#pragma unroll 4
+    for (int row = warp * rows_per_pass + sub; row < n_rows; row += 8 * rows_per_pass) {
+        const int ch = row / sg.rh, rh = row - ch * sg.rh;
+        const int ci = ci_lo + ch, ih = ih0 + rh;
+        const bool row_ok = ci < g.Cin && ih >= 0 && ih < g.H;
+        const float* src = x + (((size_t)n * g.Cin + (row_ok ? ci : 0)) * g.H + (row_ok ? ih : 0)) * g.W;
+        float* dst = region + (size_t)row * sg.rw;
+        for (int c = lc; c < sg.rw; c += lw) {
+            const int iw = iw0 + c;
+            dst[c] = (row_ok && iw >= 0 && iw < g.W) ? __ldg(src + iw) : 0.0f;
         }
     }
+    __syncthreads();
+
+    const int kql = lane & 7, tl = lane >> 3;
+    const int n_pos = sg.rt * sg.seg_w;                         // <= 256
+    const int4* koff4 = reinterpret_cast<const int4*>(koff);
+    for (int tb = warp * 4; tb < n_pos; tb += 32) {
+        const int ti = tb + tl;
+        const int po = ti < n_pos ? poff[ti] : -1;
+        if (po < 0) continue;
+        const int r = ti / sg.seg_w, c = ti - r * sg.seg_w;
+        const size_t t = ((size_t)n * g.OH + oh0 + r) * g.OW + ow0 + c;
+        for (int kq = kq0 + kql; kq < kq1; kq += 8) {
+            const int4 ko = koff4[kq - kq0];
+            float v[4];
+            v[0] = ko.x < 0 ? 0.0f : region[ko.x + po];
+            v[1] = ko.y < 0 ? 0.0f : region[ko.y + po];
+            v[2] = ko.z < 0 ? 0.0f : region[ko.z + po];
+            v[3] = ko.w < 0 ? 0.0f : region[ko.w + po];
+            store_quad_g<MODE>(V_hi, V_lo, t * g.k_pad + 4 * (size_t)kq, v);
+        }
+    }
+}
+
+// Block shape of the staged gather for a layer; false when no slab of at least 8 groups fits the shared-memory budget.
+bool plan_staged_gather(const GatherGeom& g, StagedGather* sg, size_t* smem)
+{
+    constexpr int kRegionFloats = 9216;                          // 36 KB
+    // (1x1 strided layers would stage rows and columns they never use: the element-wise gather serves them)
+    if (g.k_pad % 4 != 0 || g.k == 1) return false;
+    const int parts = (g.OW + 63) / 64;
+    sg->seg_w = (g.OW + parts - 1) / parts;
+    sg->segs = (g.OW + sg->seg_w - 1) / sg->seg_w;
+    // positions per CTA: enough for some tens of kilobytes of V per CTA when its rows are short
+    const int max_pos = g.k_pad <= 64 ? 256 : (g.k_pad <= 128 ? 128 : 64);
+    int rt = max_pos / sg->seg_w;
+    if (rt < 1) rt = 1;
+    if (rt > g.OH) rt = g.OH;
+    sg->rt = rt;
+    sg->row_tiles = (g.OH + rt - 1) / rt;
+    sg->rh = (rt - 1) * g.stride + (g.k - 1) * g.dil + 1;
+    sg->rw = (sg->seg_w - 1) * g.stride + (g.k - 1) * g.dil + 1;
+    sg->kq_n = g.k_pad / 4;
+    const int k2 = g.k * g.k;
+    const long long plane = (long long)sg->rh * sg->rw;
+    int best = 0;
+    for (int q = 8; q <= 64; q += 8) {
+        const int qq = q < sg->kq_n ? q : sg->kq_n;
+        const long long chans = (4LL * qq + k2 - 2) / k2 + 1;    // channels a slab of qq groups can touch
+        if (chans * plane <= kRegionFloats) best = qq;
+        if (qq == sg->kq_n) break;
+    }
+    if (best == 0) return false;
+    sg->slab_q = best;
+    const long long chans = (4LL * best + k2 - 2) / k2 + 1;
+    *smem = (size_t)best * 16 + 256 * 4 + (size_t)(chans * plane) * 4;
+    return true;
 }
 
 // Generic direct convolution: one thread per output element.
@@ -492,6 +622,24 @@ cudaError_t launch_gather(const float* x, void* V_hi, void* V_lo, const GatherGe
             case STORE_TF32_SPLIT: return launch_overlapped(gather_1x1_kernel<STORE_TF32_SPLIT>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
             case STORE_BF16_SPLIT: return launch_overlapped(gather_1x1_kernel<STORE_BF16_SPLIT>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
             default: return launch_overlapped(gather_1x1_kernel<STORE_FP32>, grid, dim3(256), 0, stream, x, V_hi, V_lo, g.Cin, hw, g.k_pad);
+        }
+    }
+    {
+        StagedGather sg;
+        size_t smem = 0;
+        if (plan_staged_gather(g, &sg, &smem)) {
+            const long long gx = (long long)g.N * sg.row_tiles * sg.segs;
+            const int gy = (sg.kq_n + sg.slab_q - 1) / sg.slab_q;
+            if (gx <= 2147483647ll && gy <= 65535 && smem <= 48 * 1024) {
+                const dim3 grid((unsigned)gx, (unsigned)gy);
+                switch (mode) {
+                    case STORE_TF32: return launch_overlapped(gather_staged_kernel<STORE_TF32>, grid, dim3(256), smem, stream, x, V_hi, V_lo, g, sg);
+                    case STORE_BF16: return launch_overlapped(gather_staged_kernel<STORE_BF16>, grid, dim3(256), smem, stream, x, V_hi, V_lo, g, sg);
+                    case STORE_TF32_SPLIT: return launch_overlapped(gather_staged_kernel<STORE_TF32_SPLIT>, grid, dim3(256), smem, stream, x, V_hi, V_lo, g, sg);
+                    case STORE_BF16_SPLIT: return launch_overlapped(gather_staged_kernel<STORE_BF16_SPLIT>, grid, dim3(256), smem, stream, x, V_hi, V_lo, g, sg);
+                    default: return launch_overlapped(gather_staged_kernel<STORE_FP32>, grid, dim3(256), smem, stream, x, V_hi, V_lo, g, sg);
+                }
+            }
         }
     }
     const long long bx = (T + 31) / 32;

@@ -46,7 +46,7 @@ Calibration default_calibration()
     c.c[6] = 80ll << 20;  // L2 bytes one chunk's V + M may occupy
     c.c[7] = 148;         // SMs
     c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
-    c.c[9] = 50000;       // as per flop of the direct kernel for Cin <= 4 (~20 TFLOP/s)
+    c.c[9] = 60000;       // as per flop of the direct kernel for Cin <= 4 (~17 TFLOP/s)
     return c;
 }
 
@@ -342,10 +342,11 @@ uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibrati
     const uint64_t x_bytes = 4ull * s.N * s.Cin * s.H * s.W;
     const uint64_t y_bytes = 4ull * s.N * s.Cout * s.OH * s.OW;
     const uint64_t v_bytes = T * Kp * b, u_bytes = (uint64_t)s.Cout * Kp * b;
-    // the patch gather: a transposition at about two thirds of the copy rate for 1x1 stride-1 layers, a generic
-    // element-wise gather at about a fifth of it otherwise (measured)
+    // the patch gather (measured rates): a transposition at about two thirds of the copy rate for 1x1 stride-1
+    // layers, the gather staged through shared memory at about a third of it for k > 1, the element-wise gather
+    // at about a fifth of it for strided 1x1 layers
     const bool transposer = s.k == 1 && s.stride == 1 && s.pad == 0 && (s.H * s.W) % 4 == 0;
-    const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3 : 10) / 2, 0, 0, cal);
+    const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3 : (s.k > 1 ? 6 : 10)) / 2, 0, 0, cal);
     // The contraction as the kernel schedules it: rounds of work items over the SMs, each item a serial loop
     // over blocks of K whose pace is the slower of the tensor core and the delivery of the two operand tiles
     // from L2 to one SM (about 63 GB/s measured, for either left operand).  With x as the left operand a work
@@ -359,7 +360,12 @@ uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibrati
     const uint64_t k_elems = 128 / b, k_blocks = ceil_div(Kp, k_elems);
     const uint64_t deliver_ps = (128ull * 128 + (uint64_t)bn * 128) * 16;
     const uint64_t mma_ps = 2ull * 128 * bn * k_elems * tensor_as(operand, cal) * sms / 1000000ull;
-    const uint64_t serial_as = rounds * k_blocks * (deliver_ps > mma_ps ? deliver_ps : mma_ps) * 1000000ull;
+    // an item's accumulator (128 x bn fp32) is drained at about 22 GB/s per SM while the next item's loop runs
+    // (two accumulators), with about half a microsecond of hand-over per item; the last drain is exposed
+    const uint64_t drain_ps = 128ull * bn * 4 * 45;
+    const uint64_t loop_ps = k_blocks * (deliver_ps > mma_ps ? deliver_ps : mma_ps);
+    const uint64_t item_ps = loop_ps > drain_ps + 500000 ? loop_ps : drain_ps + 500000;
+    const uint64_t serial_as = (rounds * item_ps + drain_ps) * 1000000ull;
     if (lhs_x) return kernel_ps((x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
     const uint64_t contract = kernel_ps((v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
     return gather + contract;

@@ -257,7 +257,9 @@ def test_invariants_delta_zero_and_batch_permutation(torch):
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("Cin,Cout,H,k,stride,pad,dil,N", [
     (64, 128, 14, 1, 1, 0, 1, 2), (64, 128, 28, 1, 2, 0, 1, 2), (32, 64, 15, 3, 2, 1, 1, 2),
-    (24, 40, 17, 3, 1, 2, 2, 1), (3, 64, 32, 7, 2, 3, 1, 2), (100, 36, 9, 1, 1, 0, 1, 3), (16, 300, 10, 3, 1, 1, 1, 1)])
+    (24, 40, 17, 3, 1, 2, 2, 1), (3, 64, 32, 7, 2, 3, 1, 2), (100, 36, 9, 1, 1, 0, 1, 3), (16, 300, 10, 3, 1, 1, 1, 1),
+    (3, 16, 150, 7, 2, 3, 1, 1), (80, 24, 20, 3, 2, 1, 1, 2), (6, 10, 9, 5, 1, 2, 1, 2), (8, 16, 33, 3, 1, 1, 3, 1),
+    (4, 8, 5, 3, 1, 1, 1, 3), (2, 8, 12, 2, 2, 0, 1, 2), (40, 16, 70, 3, 1, 1, 1, 1)])
 @pytest.mark.parametrize("operand", [B.OPERAND_TF32, B.OPERAND_BF16, B.OPERAND_FP32_REF])
 def test_gemm_scheme(torch, Cin, Cout, H, k, stride, pad, dil, N, operand):
     layer = W.ConvLayer("t", N, Cin, Cout, H, H, k, stride, pad, dil, relu=True, seed=Cin + Cout)
