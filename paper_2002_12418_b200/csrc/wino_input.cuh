@@ -401,6 +401,117 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
     if (*abortp) __nanosleep(200000);
 }
 
+// Small planes whose rows are not 16-byte aligned (W not a multiple of 4: 14 x 14, 7 x 7, ...), which TMA
+// cannot address row by row: one CTA per (image, block of 64 channels) copies the 64 contiguous channel planes
+// into shared memory with plain coalesced loads, each plane zero-padded to hp rows x wp columns (image row ih
+// at staged row ih + pad, image column iw at staged column lead + iw; everything else stays zero, which is the
+// convolution's padding and the overhang of the last tiles), and then transforms ALL tiles of the image from
+// there with the same row and column passes as the ring-buffer kernel: a tile's vectors are found exactly as
+// there, with wp words between staged rows.  hp and wp / 4 are odd, so that 32 lanes reading 128-bit vectors
+// from 32 consecutive planes touch every bank once.
+struct PlaneItems {
+    int hp, wp, lead, cblocks;
+};
+
+template <int ALPHA, bool SYM, bool PAIR>
+__global__ void __launch_bounds__(kItThreads, 1)
+input_transform_plane_kernel(const float* __restrict__ x, char* V_hi, char* V_lo, WinoGeom g, PlaneItems pi, int mode,
+                             const __grid_constant__ MatBt2 Bt)
+{
+    extern __shared__ __align__(128) float s_buf[];
+    using T = typename std::conditional<PAIR, float2, float>::type;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int plane = pi.hp * pi.wp;
+    {
+        float4* z = reinterpret_cast<float4*>(s_buf);
+        for (int i = threadIdx.x; i < kItChannels * plane / 4; i += kItThreads) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
+    __syncthreads();
+    const int img = blockIdx.x / pi.cblocks, cb = blockIdx.x - img * pi.cblocks;
+    const int c0 = cb * kItChannels, hw = g.H * g.W;
+    {
+        // A warp copies channels warp, warp + 16, ... (kItChannels / kItWarps of them), 32 pixels per step; the
+        // steps of all its channels form one sequence, taken eight at a time: eight loads in flight per lane,
+        // then the eight stores.  Channels beyond Cin are skipped: their planes stay zero.
+        constexpr int kChPerWarp = kItChannels / kItWarps;
+        const int steps_per_ch = (hw + 31) / 32, n_steps = kChPerWarp * steps_per_ch;
+        const float* ximg = x + (size_t)img * g.Cin * hw;
+        for (int s0 = 0; s0 < n_steps; s0 += 8) {
+            float v[8];
+            int dst[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int st = s0 + k;
+                const int cw = st / steps_per_ch, p = (st - cw * steps_per_ch) * 32 + lane;
+                const int c = warp + cw * kItWarps, ci = c0 + c;
+                const bool ok = st < n_steps && p < hw && ci < g.Cin;
+                v[k] = ok ? __ldg(ximg + (size_t)ci * hw + p) : 0.0f;
+                const int r = p / g.W, col = p - r * g.W;
+                dst[k] = ok ? slot_of<PAIR>(c) * plane + (g.pad + r) * pi.wp + pi.lead + col : -1;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (dst[k] >= 0) s_buf[dst[k]] = v[k];
+        }
+    }
+    __syncthreads();
+    const int eb = (mode == STORE_BF16 || mode == STORE_BF16_SPLIT) ? 2 : 4;
+    const long long plane_bytes = (long long)g.v_plane * eb;
+    const int units = g.th * g.tw * (PAIR ? 1 : 2);                // (tile[, half of the channel block])
+    for (int u = warp; u < units; u += kItWarps) {
+        const int ti = PAIR ? u : (u >> 1), half = PAIR ? 0 : (u & 1);
+        const int ty = ti / g.tw, tx = ti - ty * g.tw;
+        const int c = c0 + (PAIR ? 2 * lane : half * 32 + lane);
+        if (c >= g.cin_pad) continue;
+        const long long tile = ((long long)img * g.th + ty) * g.tw + tx;
+        const int s0 = pi.lead + tx * g.m - g.pad;                 // staged column of the tile's first input column
+        const float* p0 = s_buf + (size_t)(PAIR ? lane : half * 32 + lane) * plane + (size_t)(ty * g.m) * pi.wp + (s0 & ~3);
+        const float* p1 = p0 + (size_t)32 * plane;
+        T h[ALPHA][ALPHA];
+        switch (s0 & 3) {
+            case 0: rows_pass<ALPHA, SYM, 0, T>(p0, p1, pi.wp, Bt, h); break;
+            case 1: rows_pass<ALPHA, SYM, 1, T>(p0, p1, pi.wp, Bt, h); break;
+            case 2: rows_pass<ALPHA, SYM, 2, T>(p0, p1, pi.wp, Bt, h); break;
+            default: rows_pass<ALPHA, SYM, 3, T>(p0, p1, pi.wp, Bt, h); break;
+        }
+        const long long off = (tile * g.cin_pad + c) * eb;
+        char* hi = V_hi + off;
+        char* lo = V_lo ? V_lo + off : nullptr;
+        switch (mode) {
+            case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T>(h, Bt, hi, lo, plane_bytes); break;
+            case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T>(h, Bt, hi, lo, plane_bytes); break;
+            case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
+            case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
+            default: cols_pass_store<ALPHA, SYM, STORE_FP32, T>(h, Bt, hi, lo, plane_bytes); break;
+        }
+    }
+}
+
+// Padded plane shape for input_transform_plane_kernel; false when 64 planes do not fit the shared-memory budget.
+inline bool plan_plane_items(const WinoGeom& g, int alpha, PlaneItems* pi, size_t* smem)
+{
+    const int lead = (g.pad + 3) / 4 * 4;
+    int hp = (g.th - 1) * g.m + alpha;
+    if (hp < g.H + g.pad) hp = g.H + g.pad;
+    if ((hp & 1) == 0) ++hp;
+    // columns: the image, and whole 4-wide vectors up to three columns past the last tile
+    int wp = lead - g.pad + (g.tw - 1) * g.m + alpha + 3;
+    if (wp < lead + g.W) wp = lead + g.W;
+    wp = (wp + 3) / 4 * 4;
+    if (((wp / 4) & 1) == 0) wp += 4;
+    const long long bytes = (long long)kItChannels * hp * wp * 4;
+    const long long blocks = (long long)g.images * ((g.cin_pad + kItChannels - 1) / kItChannels);
+    if (bytes > kItSmemBudget || blocks > 2147483647ll) return false;
+    pi->hp = hp;
+    pi->wp = wp;
+    pi->lead = lead;
+    pi->cblocks = (g.cin_pad + kItChannels - 1) / kItChannels;
+    *smem = (size_t)bytes;
+    return true;
+}
+
 // True when Bt (alpha x alpha, row-major) has the zero pattern and the +p / -p row symmetry
 // that pass_1d<.., SYM = true> assumes.
 inline bool bt_has_symmetric_structure(const float* Bt, int alpha)
@@ -483,6 +594,21 @@ cudaError_t launch_input_ws(const float* x, void* V_hi, void* V_lo, const WinoGe
     if (tma_ok) {
         if (!plan_input_items(g, ALPHA, true, num_sms, &it) || !encode_input_map(&xmap, x, g.images, g.Cin, g.H, g.W, it.wb, kPair))
             tma_ok = false;
+    }
+    if (!tma_ok) {
+        // small planes: the whole image of a channel block in shared memory
+        PlaneItems pi;
+        size_t psmem = 0;
+        if (plan_plane_items(g, ALPHA, &pi, &psmem)) {
+            auto launch_plane = [&](auto kern) -> cudaError_t {
+                cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kItSmemBudget);
+                if (e != cudaSuccess) return e;
+                return launch_overlapped(kern, dim3((unsigned)(g.images * pi.cblocks)), dim3(kItThreads), psmem, stream, x,
+                                         static_cast<char*>(V_hi), static_cast<char*>(V_lo), g, pi, mode, bt);
+            };
+            if (sym) return launch_plane(input_transform_plane_kernel<ALPHA, true, kPair>);
+            return launch_plane(input_transform_plane_kernel<ALPHA, false, kPair>);
+        }
     }
     if (!tma_ok && !plan_input_items(g, ALPHA, false, num_sms, &it)) return cudaErrorInvalidConfiguration;
     const size_t smem = (size_t)it.nbuf * it.buf_words * sizeof(float);
