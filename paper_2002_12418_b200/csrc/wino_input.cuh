@@ -431,13 +431,41 @@ input_transform_plane_kernel(const float* __restrict__ x, char* V_hi, char* V_lo
     __syncthreads();
     const int img = blockIdx.x / pi.cblocks, cb = blockIdx.x - img * pi.cblocks;
     const int c0 = cb * kItChannels, hw = g.H * g.W;
-    {
+    const float* ximg = x + (size_t)img * g.Cin * hw;
+    if (hw <= 256) {
+        // A lane's pixels (lane, lane + 32, ...) land at the same offsets in every plane: decode them once, then
+        // copy two channels per step, sixteen loads in flight per lane.  Channels beyond Cin stay zero.
+        int off[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int p = k * 32 + lane, r = p / g.W;
+            off[k] = p < hw ? (g.pad + r) * pi.wp + pi.lead + (p - r * g.W) : -1;
+        }
+        for (int c = warp; c < kItChannels; c += 2 * kItWarps) {
+            float v[2][8];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int ci = c0 + c + j * kItWarps;
+                const float* src = ximg + (size_t)(ci < g.Cin ? ci : 0) * hw + lane;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[j][k] = (off[k] >= 0 && ci < g.Cin) ? __ldg(src + 32 * k) : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float* dst = s_buf + (size_t)slot_of<PAIR>(c + j * kItWarps) * plane;
+                if (c0 + c + j * kItWarps < g.Cin) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (off[k] >= 0) dst[off[k]] = v[j][k];
+                }
+            }
+        }
+    } else {
         // A warp copies channels warp, warp + 16, ... (kItChannels / kItWarps of them), 32 pixels per step; the
         // steps of all its channels form one sequence, taken eight at a time: eight loads in flight per lane,
         // then the eight stores.  Channels beyond Cin are skipped: their planes stay zero.
         constexpr int kChPerWarp = kItChannels / kItWarps;
         const int steps_per_ch = (hw + 31) / 32, n_steps = kChPerWarp * steps_per_ch;
-        const float* ximg = x + (size_t)img * g.Cin * hw;
         for (int s0 = 0; s0 < n_steps; s0 += 8) {
             float v[8];
             int dst[8];
