@@ -30,7 +30,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (mean over the four layers of one step) from one ncu
 # capture of this file's default workload (profiles/bench_config1_b32_launch_list.md gives the command).  Valid
 # for config1_b32 / tf32 and the kernels as captured; set an entry to None when its kernel changes.
-NCU_DRAM_BYTES_PER_LAUNCH = {"config1_b32/tf32": {"input": 40.31e6, "contraction": 45.37e6, "output": 15.48e6}}
+NCU_DRAM_BYTES_PER_LAUNCH = {"config1_b32/tf32": {"input": 40.30e6, "contraction": 45.51e6, "output": 15.49e6}}
 
 
 def workload_layers(name: str):
