@@ -197,6 +197,30 @@ def test_forced_winograd_variants(torch, m, operand, passes, cls):
         assert_close(got, ref, cls, "m=%d" % m)
 
 
+# Widths that are not a multiple of 4 (rows not 16-byte aligned) take the input transform that stages whole
+# channel planes: planes up to 256 pixels and larger ones, channel counts below, off and above the 64-channel
+# block, odd channel counts, non-square images, k = 5, and a plane too large for shared memory (33 x 33,
+# which falls back to the ring kernel).  The integer run is bit-exact for F(2x2,3x3) with unit points, whose
+# transforms are exact on small integers (entries 0, +-1, 1/2): every element of V was built from the right pixels.
+@pytest.mark.parametrize("Cin,Cout,H,W_,k,m,N", [
+    (3, 8, 14, 14, 3, 2, 2), (66, 24, 7, 7, 3, 4, 3), (130, 16, 13, 13, 3, 4, 1), (64, 32, 18, 18, 3, 6, 2),
+    (17, 20, 17, 22, 3, 2, 1), (40, 8, 10, 30, 3, 4, 2), (24, 8, 30, 10, 3, 2, 1), (5, 4, 5, 6, 3, 2, 2),
+    (32, 16, 15, 15, 5, 2, 1), (64, 16, 33, 33, 3, 4, 1)])
+def test_winograd_on_planes_with_unaligned_rows(torch, Cin, Cout, H, W_, k, m, N):
+    layer = W.ConvLayer("t", N, Cin, Cout, H, W_, k, 1, (k - 1) // 2, relu=True, seed=Cin + H + W_)
+    x, w, b = W.make_inputs(layer)
+    o = opts_for(layer, force_algo=B.ALGO_WINOGRAD, force_m=m, operand=B.OPERAND_BF16, passes=3)
+    got, info, _ = run_layer(torch, layer, o, (x, w, b))
+    assert info.algo == B.ALGO_WINOGRAD and info.m == m
+    assert_close(got, oracle(layer, x, w, b), B.PREC_TF32, "winograd, unaligned rows")
+    if m == 2 and k == 3:
+        xi, wi, bi = W.integer_inputs(layer, -2, 2)
+        oi = opts_for(layer, force_algo=B.ALGO_WINOGRAD, force_m=2, operand=B.OPERAND_TF32, passes=1,
+                      points_id=B.POINTS_UNIT)
+        goti, _, _ = run_layer(torch, layer, oi, (xi, wi, bi))
+        assert np.array_equal(goti.astype(np.float64), oracle(layer, xi, wi, bi))
+
+
 @pytest.mark.parametrize("batch", [1, 3])
 def test_config1_planner_choice(torch, batch):
     for layer in W.config1(1):
