@@ -536,9 +536,14 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
     const bool col_ok = plane_ok && icol0 >= 0 && icol0 < g.W;            // the whole vector lies inside or outside
     const bool owns = col_ok && (ls >= 1 || strips == 1) && (STRIDE == 2 || ls <= SW - 2 || strip == strips - 1);
     const int ocol0 = STRIDE == 1 ? icol0 : icol0 / 2;
+    // Rows are addressed by running pointers (one 32-bit multiply per loaded row, none per stored row); the row
+    // registers rotate unconditionally and only the store of a row past the band is suppressed, so that the
+    // unrolled loop needs no register moves.
+    const float* xcol = xp + (col_ok ? icol0 : 0);
+    const int Hd = g.H, Wd = g.W, OWd = g.OW;
     auto load = [&](int ih, DwRow<VIN>& r) {
-        const bool ok = col_ok && ih >= 0 && ih < g.H;
-        dw_load_row<VIN>(xp + (size_t)(ok ? ih : 0) * g.W + (ok ? icol0 : 0), ok, r);
+        const bool ok = col_ok && (unsigned)ih < (unsigned)Hd;
+        dw_load_row<VIN>(xcol + (ok ? ih * Wd : 0), ok, r);
     };
     auto edges = [&](DwRow<VIN>& r) {                                      // neighbours' border values
         const float l = __shfl_up_sync(full, r.e[VIN], 1, SW);
@@ -548,7 +553,8 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
             r.e[VIN + 1] = ls == SW - 1 ? 0.0f : q;
         }
     };
-    auto out = [&](int oh, const DwRow<VIN>& a, const DwRow<VIN>& m, const DwRow<VIN>& z) {
+    const bool relu = g.relu != 0;
+    auto out = [&](float* q, bool store, const DwRow<VIN>& a, const DwRow<VIN>& m, const DwRow<VIN>& z) {
         float acc[VOUT];
 #pragma unroll
         for (int j = 0; j < VOUT; ++j) {
@@ -559,15 +565,19 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
                 v = fmaf(wk[3 + t], m.e[STRIDE * j + t], v);
                 v = fmaf(wk[6 + t], z.e[STRIDE * j + t], v);
             }
-            acc[j] = g.relu ? fmaxf(v, 0.0f) : v;
+            acc[j] = v;
         }
-        if (owns) {
-            float* q = yp + (size_t)oh * g.OW + ocol0;
+        if (relu) {
+#pragma unroll
+            for (int j = 0; j < VOUT; ++j) acc[j] = fmaxf(acc[j], 0.0f);
+        }
+        if (store) {
             if (VOUT == 4) *reinterpret_cast<float4*>(q) = make_float4(acc[0], acc[1], acc[2], acc[VOUT - 1]);
             else if (VOUT == 2) *reinterpret_cast<float2*>(q) = make_float2(acc[0], acc[VOUT - 1]);
             else *q = acc[0];
         }
     };
+    float* yrow = yp + (owns ? oh0 * OWd + ocol0 : 0);                     // output row oh0 of this lane's columns
 
     if (STRIDE == 1) {
         DwRow<VIN> r0, r1;
@@ -581,13 +591,12 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
             for (int k = 0; k < 4; ++k) load(oh + k + 1, nx[k]);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                if (oh + k < oh1) {
-                    edges(nx[k]);
-                    out(oh + k, r0, r1, nx[k]);
-                    r0 = r1;
-                    r1 = nx[k];
-                }
+                edges(nx[k]);
+                out(yrow + k * OWd, owns && oh + k < oh1, r0, r1, nx[k]);
+                r0 = r1;
+                r1 = nx[k];
             }
+            yrow += 4 * OWd;
         }
     } else {
         DwRow<VIN> prev;
@@ -600,9 +609,10 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
             load(2 * oh + 2, rc);
             load(2 * oh + 3, rd);
             edges(ra); edges(rb); edges(rc); edges(rd);
-            out(oh, prev, ra, rb);
-            if (oh + 1 < oh1) out(oh + 1, rb, rc, rd);
+            out(yrow, owns, prev, ra, rb);
+            out(yrow + OWd, owns && oh + 1 < oh1, rb, rc, rd);
             prev = rd;
+            yrow += 2 * OWd;
         }
     }
 }
