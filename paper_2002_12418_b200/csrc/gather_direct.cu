@@ -512,14 +512,15 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
     constexpr int PPW = 32 / SW;                      // planes per warp
     constexpr int VOUT = STRIDE == 1 ? VIN : VIN / 2;
     const int lane = threadIdx.x & 31, ls = lane % SW, seg = lane / SW;
-    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (plane group, band, strip)
-    if (unit >= n_units) return;
-    const int strip = (int)(unit % strips);
-    const long long rest = unit / strips;
-    const int band = (int)(rest % bands);
-    const long long plane = (rest / bands) * PPW + seg;
-    const bool plane_ok = plane < n_planes;
-    const int c = (int)((plane_ok ? plane : 0) % g.Cout);
+    // (plane group, band, strip) in 32-bit arithmetic: the launcher refuses more than 2^31 - 1 units
+    const unsigned unit = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if ((long long)unit >= n_units) return;
+    const int strip = (int)(unit % (unsigned)strips);
+    const unsigned rest = unit / (unsigned)strips;
+    const int band = (int)(rest % (unsigned)bands);
+    const unsigned plane = (rest / (unsigned)bands) * PPW + seg;
+    const bool plane_ok = (long long)plane < n_planes;
+    const int c = (int)((plane_ok ? plane : 0u) % (unsigned)g.Cout);
     const float* xp = x + (size_t)(plane_ok ? plane : 0) * g.H * g.W;
     float* yp = y + (size_t)(plane_ok ? plane : 0) * g.OH * g.OW;
     float wk[9];
@@ -684,7 +685,7 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
             const long long groups = (planes + 32 / sw - 1) / (32 / sw);
             const long long units = groups * strips * bands;
             const long long blocks = (units + 3) / 4;
-            if (blocks > 2147483647ll) return cudaErrorInvalidValue;
+            if (units > 2147483647ll - 4) return cudaErrorInvalidValue;
 #define MNNB_DWV_LAUNCH(ST, SWV, VI) depthwise3x3_vec_kernel<ST, SWV, VI><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, planes, units)
 #define MNNB_DWV_PICK(ST, VI) do { if (sw == 8) MNNB_DWV_LAUNCH(ST, 8, VI); else if (sw == 16) MNNB_DWV_LAUNCH(ST, 16, VI); else MNNB_DWV_LAUNCH(ST, 32, VI); } while (0)
             if (g.stride == 1) {
