@@ -422,17 +422,16 @@ __global__ void __launch_bounds__(128) depthwise3x3_kernel(const float* __restri
             for (int k = 0; k < 4; ++k) nx[k] = row(oh + k + 1);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                if (oh + k < oh1) {
-                    const float r2 = nx[k];
-                    const float l2 = __shfl_up_sync(full, r2, 1, SW), q2 = right(r2);
-                    float acc = b;
-                    acc = fmaf(wk[0], l0, acc); acc = fmaf(wk[1], r0, acc); acc = fmaf(wk[2], q0, acc);
-                    acc = fmaf(wk[3], l1, acc); acc = fmaf(wk[4], r1, acc); acc = fmaf(wk[5], q1, acc);
-                    acc = fmaf(wk[6], l2, acc); acc = fmaf(wk[7], r2, acc); acc = fmaf(wk[8], q2, acc);
-                    if (out_ok) yp[(size_t)(oh + k) * g.OW + ow] = g.relu ? fmaxf(acc, 0.0f) : acc;
-                    l0 = l1; r0 = r1; q0 = q1;
-                    l1 = l2; r1 = r2; q1 = q2;
-                }
+                // (rows past the band are computed and not stored, so that the row registers rotate unconditionally)
+                const float r2 = nx[k];
+                const float l2 = __shfl_up_sync(full, r2, 1, SW), q2 = right(r2);
+                float acc = b;
+                acc = fmaf(wk[0], l0, acc); acc = fmaf(wk[1], r0, acc); acc = fmaf(wk[2], q0, acc);
+                acc = fmaf(wk[3], l1, acc); acc = fmaf(wk[4], r1, acc); acc = fmaf(wk[5], q1, acc);
+                acc = fmaf(wk[6], l2, acc); acc = fmaf(wk[7], r2, acc); acc = fmaf(wk[8], q2, acc);
+                if (out_ok && oh + k < oh1) yp[(size_t)(oh + k) * g.OW + ow] = g.relu ? fmaxf(acc, 0.0f) : acc;
+                l0 = l1; r0 = r1; q0 = q1;
+                l1 = l2; r1 = r2; q1 = q2;
             }
         }
     } else {
