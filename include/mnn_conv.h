@@ -90,6 +90,11 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
  *              the low 13 mantissa bits of x (truncation) instead of a rounded copy being
  *              stored.  AUTO = the planner takes the cheaper where X applies.  Asking
  *              for X where it does not apply fails the plan.
+ *   fused      Winograd F(2x2, 3x3) as ONE kernel (input transform, contraction and output
+ *              transform fused; the transformed tensors V and M never reach device memory):
+ *              0 = the planner weighs it against the other candidates, 1 = never,
+ *              2 = this kernel or fail.  It applies to 3x3 stride-1 undilated ungrouped layers with
+ *              Cin a multiple of 8 and pad <= 2, accuracy class permitting single-pass TF32 at m = 2.
  */
 typedef struct {
     int groups;
@@ -102,7 +107,8 @@ typedef struct {
     int points_id;
     int chunk_images;
     int gemm_lhs;
-    int reserved[6];
+    int fused;
+    int reserved[5];
 } mnn_conv_opts;
 
 /*
@@ -110,8 +116,13 @@ typedef struct {
  * cost = sum over its kernels of max(bytes * c_byte, tensor flops * c_tensor,
  * ALU flops * c_alu) + launch cost, in integer picoseconds).
  * cost_ps[] order: 0 DIRECT; 1 GEMM tf32; 2 GEMM bf16; 3..5 Winograd m=2,4,6 tf32x1;
- * 6..8 tf32x3; 9..11 bf16x1; 12..14 bf16x3; 15 unused.  Candidates that are not
- * applicable or fail the accuracy gate hold MNN_COST_INADMISSIBLE.
+ * 6..8 tf32x3; 9..11 bf16x1; 12..14 bf16x3; 15 Winograd F(2x2,3x3) tf32x1 as one fused kernel.
+ * Candidates that are not applicable or fail the accuracy gate hold MNN_COST_INADMISSIBLE; every
+ * other figure saturates at MNN_COST_INADMISSIBLE - 1.
+ * paper_mul[] is the paper's own multiplication count (Eq. 2) for output tile sizes n = 1, 2, 4, 6,
+ * read as a count per tile (so multiplied by the number of tiles) with the output-channel factor
+ * its third term lacks as printed; paper_n_hat is its argmin (1 = sliding window, Eq. 3).  It is
+ * reported for comparison only and does not enter the choice.
  * Workspace layout (byte offsets from the workspace base, each 1024-aligned):
  *   u_offset  transformed weights  U [alpha^2][Cout][cin_pad]  (operand format; hi then lo when passes = 3)
  *   v_offset  transformed inputs   V [alpha^2][chunk_tiles][cin_pad] of one chunk (same format)
@@ -130,6 +141,9 @@ typedef struct {
     int chosen_candidate;            /* index into cost_ps, -1 when the choice was forced outside the list */
     int gemm_lhs;                    /* GEMM scheme: MNN_GEMM_LHS_PATCHES or MNN_GEMM_LHS_X as planned, else 0 */
     unsigned long long cost_ps[MNN_N_CANDIDATES];
+    int fused;                       /* 1 when the plan is the single fused Winograd kernel (no V, no M) */
+    int paper_n_hat;
+    unsigned long long paper_mul[4];
 } mnn_conv_info;
 
 /* Plan one layer with groups = 1, relu = 1, accuracy class TF32, everything else
@@ -243,7 +257,11 @@ MNN_API long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int
  * consts[8] attoseconds per flop of the direct kernel
  * consts[9] attoseconds per flop of the direct kernel for layers with at most 4 input channels
  *           (0 = use consts[8])
- * consts[10..15] reserved (0).
+ * consts[10] attoseconds per byte of transformed weights delivered from L2 to ONE SM (fused Winograd kernel)
+ * consts[11] picoseconds the fused kernel's tensor work takes per block of 32 input channels of one work item
+ * consts[12] picoseconds of epilogue per work item of the fused kernel
+ *            (consts[10] or [11] = 0: the fused kernel is never chosen by the planner)
+ * consts[13..15] reserved (0).
  * mnn_calibrate measures them on the current device (launches micro-benchmarks and
  * synchronises; allocates and frees its own scratch) and installs them;
  * mnn_set_calibration installs a frozen record so that plans are reproducible;

@@ -18,6 +18,7 @@ PREC_TF32, PREC_BF16 = 0, 1
 OPERAND_AUTO, OPERAND_TF32, OPERAND_BF16, OPERAND_FP32_REF = 0, 1, 2, 3
 POINTS_AUTO, POINTS_PAPER, POINTS_UNIT, POINTS_MIXED = 0, 1, 2, 3
 GEMM_LHS_AUTO, GEMM_LHS_PATCHES, GEMM_LHS_X = 0, 1, 2
+FUSED_AUTO, FUSED_NEVER, FUSED_ONLY = 0, 1, 2
 STAGE_WEIGHT, STAGE_INPUT, STAGE_CONTRACT, STAGE_OUTPUT, STAGE_ALL = 1, 2, 4, 8, 15
 N_CANDIDATES, N_CONSTS = 16, 16
 COST_INADMISSIBLE = 0xFFFFFFFFFFFFFFFF
@@ -37,7 +38,7 @@ class ConvOpts(ctypes.Structure):
     _fields_ = [("groups", ctypes.c_int), ("relu", ctypes.c_int), ("precision", ctypes.c_int),
                 ("operand", ctypes.c_int), ("passes", ctypes.c_int), ("force_algo", ctypes.c_int),
                 ("force_m", ctypes.c_int), ("points_id", ctypes.c_int), ("chunk_images", ctypes.c_int),
-                ("gemm_lhs", ctypes.c_int), ("reserved", ctypes.c_int * 6)]
+                ("gemm_lhs", ctypes.c_int), ("fused", ctypes.c_int), ("reserved", ctypes.c_int * 5)]
 
 
 class ConvInfo(ctypes.Structure):
@@ -52,7 +53,8 @@ class ConvInfo(ctypes.Structure):
                 ("m_offset", ctypes.c_longlong), ("m_bytes", ctypes.c_longlong),
                 ("predicted_error_ppm", ctypes.c_longlong),
                 ("chosen_candidate", ctypes.c_int), ("gemm_lhs", ctypes.c_int),
-                ("cost_ps", ctypes.c_ulonglong * N_CANDIDATES)]
+                ("cost_ps", ctypes.c_ulonglong * N_CANDIDATES),
+                ("fused", ctypes.c_int), ("paper_n_hat", ctypes.c_int), ("paper_mul", ctypes.c_ulonglong * 4)]
 
 
 class LayerDesc(ctypes.Structure):
@@ -153,11 +155,12 @@ def _check(rc: int) -> None:
 
 
 def make_opts(groups=1, relu=0, precision=PREC_TF32, operand=0, passes=0, force_algo=0, force_m=0, points_id=0,
-              chunk_images=0, gemm_lhs=0) -> ConvOpts:
+              chunk_images=0, gemm_lhs=0, fused=0) -> ConvOpts:
     o = ConvOpts()
     o.groups, o.relu, o.precision, o.operand, o.passes = groups, int(bool(relu)), precision, operand, passes
     o.force_algo, o.force_m, o.points_id, o.chunk_images = force_algo, force_m, points_id, chunk_images
     o.gemm_lhs = gemm_lhs
+    o.fused = fused
     return o
 
 

@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmnnconv_b200.so")
-SOURCES = ["api.cu", "calibrate.cu", "contract_umma.cu", "gather_direct.cu", "wino_transforms.cu", "wino_inst_k2.cu", "wino_inst_a4_6.cu",
+SOURCES = ["api.cu", "calibrate.cu", "contract_umma.cu", "wino_fused.cu", "gather_direct.cu", "wino_transforms.cu", "wino_inst_k2.cu", "wino_inst_a4_6.cu",
            "wino_inst_a8.cu", "wino_inst_a10.cu", "wino_inst_a12.cu",
            "generator.cpp", "planner.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -27,26 +27,36 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def _headers_mtime() -> float:
-    newest = os.path.getmtime(os.path.abspath(__file__))
-    for root in (CSRC, os.path.join(os.path.dirname(HERE), "include")):
-        for name in os.listdir(root):
-            if name.endswith((".h", ".cuh")):
-                newest = max(newest, os.path.getmtime(os.path.join(root, name)))
-    return newest
+def _local_includes(path: str, seen: set) -> None:
+    """Collects, recursively, the files `path` includes with quotes (headers of this repo only)."""
+    if path in seen or not os.path.exists(path):
+        return
+    seen.add(path)
+    with open(path, errors="replace") as f:
+        for line in f:
+            s = line.strip()
+            if s.startswith("#include \""):
+                name = s.split('"')[1]
+                _local_includes(os.path.normpath(os.path.join(os.path.dirname(path), name)), seen)
+
+
+def _newest_dependency(src: str) -> float:
+    """mtime of the newest of the source and every repo header it reaches (after a change of the compiler
+    flags in this file, build with --force)."""
+    seen: set = set()
+    _local_includes(os.path.join(CSRC, src), seen)
+    return max(os.path.getmtime(p) for p in seen)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(BUILD, exist_ok=True)
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
-    hdr = _headers_mtime()
     rebuilt = []
 
     def compile_one(src: str) -> str:
         obj = os.path.join(BUILD, os.path.splitext(src)[0] + ".o")
-        if (not force and os.path.exists(obj)
-                and os.path.getmtime(obj) >= max(hdr, os.path.getmtime(os.path.join(CSRC, src)))):
+        if not force and os.path.exists(obj) and os.path.getmtime(obj) >= _newest_dependency(src):
             return obj
         rebuilt.append(src)
         cmd = [nvcc] + NVCC_FLAGS + extra + ["-x", "cu", "-c", os.path.join(CSRC, src), "-o", obj]

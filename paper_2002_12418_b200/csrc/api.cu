@@ -55,6 +55,8 @@ struct mnn_conv_plan_s {
     long long ws_bytes = 0;
     const float* prepared_w = nullptr;
     UmmaContract uc;
+    bool fused = false;              // Winograd F(2x2,3x3) as the single fused kernel: the workspace holds U only
+    FusedWino fw;
     // optional per-launch timing
     bool profiling = false;
     std::vector<cudaEvent_t> events;     // pairs (before, after)
@@ -100,9 +102,10 @@ void layout_workspace(mnn_conv_plan_t p)
         p->chunk_tiles = (long long)d.chunk_images * th * tw;
         p->m_row_stride = (int)align_up(p->chunk_tiles, 32);
         p->u_bytes = align_up(a2 * s.Cout * p->cin_pad * eb, 2048);
-        p->v_bytes = align_up(a2 * p->chunk_tiles * p->cin_pad * eb, 2048);
-        p->m_bytes = align_up(a2 * s.Cout * p->m_row_stride * 4, 1024);
-        p->launches_per_run = 3 * d.n_chunks;
+        p->fused = d.fused != 0;
+        p->v_bytes = p->fused ? 0 : align_up(a2 * p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->m_bytes = p->fused ? 0 : align_up(a2 * s.Cout * p->m_row_stride * 4, 1024);
+        p->launches_per_run = p->fused ? 1 : 3 * d.n_chunks;
     } else {
         p->cin_pad = (int)align_up((long long)s.Cin * s.k * s.k, 8);
         p->chunk_tiles = (long long)s.N * s.OH * s.OW;
@@ -182,7 +185,7 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
     }
     if (o.operand < 0 || o.operand > MNN_OPERAND_FP32_REF || !(o.passes == 0 || o.passes == 1 || o.passes == 3) ||
         o.force_algo < 0 || o.force_algo > MNN_ALGO_DIRECT || o.points_id < 0 || o.points_id > MNN_POINTS_MIXED ||
-        o.force_m < 0 || o.chunk_images < 0) {
+        o.force_m < 0 || o.chunk_images < 0 || o.gemm_lhs < 0 || o.gemm_lhs > MNN_GEMM_LHS_X || o.fused < 0 || o.fused > 2) {
         fail(MNN_EINVAL, "an option is outside its range");
         return nullptr;
     }
@@ -275,7 +278,20 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     info->chosen_candidate = p->d.chosen;
     info->gemm_lhs = p->d.algo == MNN_ALGO_GEMM ? p->d.gemm_lhs : 0;
     for (int i = 0; i < MNN_N_CANDIDATES; ++i) info->cost_ps[i] = p->d.cost_ps[i];
+    info->fused = p->fused ? 1 : 0;
+    info->paper_n_hat = p->d.paper_n_hat;
+    for (int i = 0; i < 4; ++i) info->paper_mul[i] = p->d.paper_mul[i];
     return MNN_OK;
+}
+
+// Tensor maps and launch parameters of the plan's tensor-core kernel for the workspace now in p->ws / p->tws.
+static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
+{
+    const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
+    if (p->fused) return fused_wino_setup(&p->fw, p->s.Cout, p->cin_pad, u_hi(p), why);
+    if (p->gemm_x) return umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), why);
+    return umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
+                               v_lo(p), why);
 }
 
 // Workspace in two parts (used by the network plan): `persistent` holds the status word and U
@@ -329,12 +345,7 @@ static int set_workspace_split(mnn_conv_plan_t p, void* persistent, long long pe
     if (e != cudaSuccess) return fail_cuda(e, "clearing the status word");
     if (p->d.operand != MNN_OPERAND_FP32_REF) {
         const char* why = "";
-        const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
-        if (p->gemm_x)
-            e = umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), &why);
-        else
-            e = umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p),
-                                    v_hi(p), v_lo(p), &why);
+        e = setup_tensor_kernels(p, &why);
         if (e != cudaSuccess) {
             p->ws = nullptr;
             return fail(MNN_ECUDA, std::string("tensor-core contraction setup: ") + why + " (" + cudaGetErrorString(e) + ")");
@@ -349,13 +360,21 @@ static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, con
     if ((mask & ~(unsigned)MNN_STAGE_ALL) || mask == 0) return fail(MNN_EINVAL, "bad stage mask");
     if (p->workspace_bytes > 0 && !p->ws) return fail(MNN_EWORKSPACE, "call mnn_conv_set_workspace first");
     const bool direct = p->d.algo == MNN_ALGO_DIRECT;
-    const bool need_x = direct || (mask & MNN_STAGE_INPUT) || (p->gemm_x && (mask & MNN_STAGE_CONTRACT));
+    const bool one_kernel = p->gemm_x || p->fused;       // x in, y out in the contraction stage
+    const bool need_x = direct || (!one_kernel && (mask & MNN_STAGE_INPUT)) || (one_kernel && (mask & MNN_STAGE_CONTRACT));
     const bool need_w = direct || (mask & MNN_STAGE_WEIGHT);
-    const bool need_y = direct || (mask & MNN_STAGE_OUTPUT) || (p->d.algo == MNN_ALGO_GEMM && (mask & MNN_STAGE_CONTRACT));
+    const bool need_y = direct || (!p->fused && (mask & MNN_STAGE_OUTPUT)) ||
+                        ((p->d.algo == MNN_ALGO_GEMM || p->fused) && (mask & MNN_STAGE_CONTRACT));
     if ((need_x && !x) || (need_w && !w) || (need_y && !y)) return fail(MNN_EINVAL, "NULL tensor pointer");
     if ((x && !aligned16(x)) || (w && !aligned16(w)) || (y && !aligned16(y)))
         return fail(MNN_EALIGN, "x, w and y must be 16-byte aligned");
-    if (x && y && (const void*)x == (const void*)y) return fail(MNN_EINVAL, "y must not alias x");
+    if (x && y) {
+        // the tensors may not overlap anywhere: a kernel reads x while another block already writes y
+        const uintptr_t x0 = reinterpret_cast<uintptr_t>(x), y0 = reinterpret_cast<uintptr_t>(y);
+        const uintptr_t x1 = x0 + 4ull * p->s.N * p->s.Cin * p->s.H * p->s.W;
+        const uintptr_t y1 = y0 + 4ull * p->s.N * p->s.Cout * p->s.OH * p->s.OW;
+        if (x0 < y1 && y0 < x1) return fail(MNN_EINVAL, "y must not overlap x");
+    }
     return MNN_OK;
 }
 
@@ -436,9 +455,24 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
         return MNN_OK;
     }
 
-    // Winograd: the three stages chunk by chunk, so that one chunk's V and M stay in L2.
     const int th = (s.OH + d.m - 1) / d.m, tw = (s.OW + d.m - 1) / d.m;
     const int alpha2 = d.alpha * d.alpha;
+    if (p->fused) {
+        // one kernel does the three stages; it is booked as the contraction stage
+        if (!(mask & MNN_STAGE_CONTRACT)) return MNN_OK;
+        WinoGeom g;
+        g.images = s.N;
+        g.Cin = s.Cin; g.Cout = s.Cout; g.H = s.H; g.W = s.W; g.OH = s.OH; g.OW = s.OW; g.k = s.k; g.pad = s.pad;
+        g.m = d.m; g.alpha = d.alpha; g.th = th; g.tw = tw; g.cin_pad = p->cin_pad;
+        g.tiles = (long long)s.N * th * tw;
+        g.v_plane = 0;
+        g.m_row_stride = 0;
+        LaunchTimer lt(p, st, 2);
+        e = launch_fused_wino(p->fw, x, bias, y, g, s.relu, p->mats, status_word(p), st);
+        if (e != cudaSuccess) return fail_cuda(e, "fused Winograd kernel");
+        return MNN_OK;
+    }
+    // Winograd: the three stages chunk by chunk, so that one chunk's V and M stay in L2.
     for (int n0 = 0; n0 < s.N; n0 += d.chunk_images) {
         const int n_img = (s.N - n0) < d.chunk_images ? (s.N - n0) : d.chunk_images;
         WinoGeom g;
@@ -819,13 +853,7 @@ extern "C" int mnn_conv_run_static(mnn_conv_plan_t p, const float* x, const floa
         if (e != cudaSuccess) return fail_cuda(e, "clearing the status word");
         if (local.d.operand != MNN_OPERAND_FP32_REF) {
             const char* why = "";
-            const int alpha2 = local.d.algo == MNN_ALGO_WINOGRAD ? local.d.alpha * local.d.alpha : 1;
-            if (local.gemm_x)
-                e = umma_contract_setup_x(&local.uc, local.s.Cout, local.s.Cin, local.cin_pad, local.s.N,
-                                          local.s.H * local.s.W, u_hi(&local), &why);
-            else
-                e = umma_contract_setup(&local.uc, local.store_mode, alpha2, local.s.Cout, local.cin_pad, local.chunk_tiles,
-                                        u_hi(&local), u_lo(&local), v_hi(&local), v_lo(&local), &why);
+            e = setup_tensor_kernels(&local, &why);
             if (e != cudaSuccess)
                 return fail(MNN_ECUDA, std::string("tensor-core contraction setup: ") + why + " (" + cudaGetErrorString(e) + ")");
         }

@@ -357,18 +357,19 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 EncodeTiledFn get_encode_fn()
 {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    // looked up once; the initialisation of a function-local static is thread-safe
+    static const EncodeTiledFn fn = [] {
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
+            return reinterpret_cast<EncodeTiledFn>(sym);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
+
+}  // namespace
 
 // 3-D map over [planes][rows][k] (k contiguous), box = [1][box_rows][128 bytes of k], 128-byte swizzle.
 bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
@@ -385,8 +386,6 @@ bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long 
                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
-
-}  // namespace
 
 namespace wino {
 // Tensor map over x [images][C][H][W] (fp32) for the input transform's row copies, no swizzle; elements

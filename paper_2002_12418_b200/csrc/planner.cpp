@@ -29,7 +29,13 @@ bool g_cal_set = false;
 uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
 constexpr uint64_t kMaxChunkBytes = 4ull << 30;   // V + M of one chunk
 uint64_t round_up(uint64_t a, uint64_t b) { return ceil_div(a, b) * b; }
-uint64_t max3(uint64_t a, uint64_t b, uint64_t c) { return a > b ? (a > c ? a : c) : (b > c ? b : c); }
+// Attosecond products of byte or flop counts and rate constants can pass 2^64 for very large layers; they
+// are formed in 128 bits and every picosecond figure saturates just below the "inadmissible" marker, so a
+// huge layer can never wrap around into a small cost.
+typedef unsigned __int128 u128;
+constexpr uint64_t kCostSaturated = MNN_COST_INADMISSIBLE - 1;
+uint64_t saturate(u128 v) { return v > (u128)kCostSaturated ? kCostSaturated : (uint64_t)v; }
+u128 max3(u128 a, u128 b, u128 c) { return a > b ? (a > c ? a : c) : (b > c ? b : c); }
 }  // namespace
 
 Calibration default_calibration()
@@ -47,6 +53,9 @@ Calibration default_calibration()
     c.c[7] = 148;         // SMs
     c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
     c.c[9] = 60000;       // as per flop of the direct kernel for Cin <= 4 (~17 TFLOP/s)
+    c.c[10] = 8000;       // as per byte of U delivered from L2 to one SM by the fused kernel (~125 GB/s per SM)
+    c.c[11] = 1300000;    // ps of tensor work per 32-channel block of a fused work item (64 MMAs of 128 x 32 x 8)
+    c.c[12] = 1500000;    // ps of epilogue per fused work item
     return c;
 }
 
@@ -282,9 +291,9 @@ int best_points(int m, int k, int operand, int passes, long long* ppm_out)
 // ---------------------------------------------------------------------------
 namespace {
 
-uint64_t kernel_ps(uint64_t as_mem, uint64_t as_tensor, uint64_t as_alu, const Calibration& cal)
+uint64_t kernel_ps(u128 as_mem, u128 as_tensor, u128 as_alu, const Calibration& cal)
 {
-    return max3(as_mem, as_tensor, as_alu) / 1000000ull + (uint64_t)cal.c[5];
+    return saturate(max3(as_mem, as_tensor, as_alu) / 1000000u + (u128)cal.c[5]);
 }
 
 uint64_t operand_bytes(int operand) { return operand == MNN_OPERAND_BF16 ? 2 : 4; }
@@ -300,7 +309,7 @@ uint64_t direct_cost(const LayerShape& s, const Calibration& cal)
     const bool stem = s.groups == 1 && s.Cin <= 4 && cal.c[9] > 0 &&
                       (long long)s.Cin * s.k * s.k * ((s.Cout + 31) / 32 * 32) * 4 <= 160 * 1024 && s.N <= 65535;
     const uint64_t rate = (uint64_t)(stem ? cal.c[9] : cal.c[8]);
-    return kernel_ps((x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, flops * rate, cal);
+    return kernel_ps((u128)(x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, (u128)flops * rate, cal);
 }
 
 }  // namespace
@@ -346,7 +355,7 @@ uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibrati
     // layers, the gather staged through shared memory at about a third of it for k > 1, the element-wise gather
     // at about a fifth of it for strided 1x1 layers
     const bool transposer = s.k == 1 && s.stride == 1 && s.pad == 0 && (s.H * s.W) % 4 == 0;
-    const uint64_t gather = kernel_ps((x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3 : (s.k > 1 ? 6 : 10)) / 2, 0, 0, cal);
+    const uint64_t gather = kernel_ps((u128)(x_bytes + v_bytes) * (uint64_t)cal.c[0] * (transposer ? 3u : (s.k > 1 ? 6u : 10u)) / 2u, 0, 0, cal);
     // The contraction as the kernel schedules it: rounds of work items over the SMs, each item a serial loop
     // over blocks of K whose pace is the slower of the tensor core and the delivery of the two operand tiles
     // from L2 to one SM (about 63 GB/s measured, for either left operand).  With x as the left operand a work
@@ -359,16 +368,16 @@ uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibrati
     const uint64_t rounds = ceil_div(tile_blocks * (uint64_t)n_co_blocks, (uint64_t)sms);
     const uint64_t k_elems = 128 / b, k_blocks = ceil_div(Kp, k_elems);
     const uint64_t deliver_ps = (128ull * 128 + (uint64_t)bn * 128) * 16;
-    const uint64_t mma_ps = 2ull * 128 * bn * k_elems * tensor_as(operand, cal) * sms / 1000000ull;
+    const uint64_t mma_ps = saturate((u128)(2ull * 128 * bn * k_elems) * tensor_as(operand, cal) * (uint64_t)sms / 1000000u);
     // an item's accumulator (128 x bn fp32) is drained at about 22 GB/s per SM while the next item's loop runs
     // (two accumulators), with about half a microsecond of hand-over per item; the last drain is exposed
     const uint64_t drain_ps = 128ull * bn * 4 * 45;
     const uint64_t loop_ps = k_blocks * (deliver_ps > mma_ps ? deliver_ps : mma_ps);
     const uint64_t item_ps = loop_ps > drain_ps + 500000 ? loop_ps : drain_ps + 500000;
-    const uint64_t serial_as = (rounds * item_ps + drain_ps) * 1000000ull;
-    if (lhs_x) return kernel_ps((x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
-    const uint64_t contract = kernel_ps((v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
-    return gather + contract;
+    const u128 serial_as = ((u128)rounds * item_ps + drain_ps) * 1000000u;
+    if (lhs_x) return kernel_ps((u128)(x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
+    const uint64_t contract = kernel_ps((u128)(v_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
+    return saturate((u128)gather + contract);
 }
 
 uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes, uint64_t n, bool resident,
@@ -387,16 +396,55 @@ uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes
     const uint64_t c0 = (uint64_t)cal.c[0], cA = (uint64_t)cal.c[4];
     // from alpha = 8 on a lane of the input transform holds one channel instead of a packed pair (twice the ALU
     // time); from alpha = 10 on the tile no longer fits the register file (measured about twice that again)
-    const uint64_t in_alu = (alpha >= 10 ? 4ull : (alpha >= 8 ? 2ull : 1ull)) * 4ull * alpha * a2 * n * tiles_img * s.Cin * cA;
-    const uint64_t in = kernel_ps(x_bytes * c0 + v_bytes * cV, 0, in_alu, cal);
-    const uint64_t con = kernel_ps((v_bytes + m_bytes) * cV + u_bytes * c0,
-                                   2ull * a2 * s.Cout * Cp * n * tiles_img * passes * tensor_as(operand, cal), 0, cal);
-    const uint64_t out = kernel_ps(m_bytes * cV + y_bytes * c0, 0,
-                                   2ull * m * alpha * (alpha + m) * n * tiles_img * s.Cout * cA, cal);
-    return in + con + out;
+    const u128 tile_channels_in = (u128)n * tiles_img * (uint64_t)s.Cin, tile_channels_out = (u128)n * tiles_img * (uint64_t)s.Cout;
+    const u128 in_alu = (alpha >= 10 ? 4u : (alpha >= 8 ? 2u : 1u)) * 4u * alpha * a2 * tile_channels_in * cA;
+    const uint64_t in = kernel_ps((u128)x_bytes * c0 + (u128)v_bytes * cV, 0, in_alu, cal);
+    const uint64_t con = kernel_ps((u128)(v_bytes + m_bytes) * cV + (u128)u_bytes * c0,
+                                   2u * a2 * Cp * tile_channels_out * (uint64_t)passes * tensor_as(operand, cal), 0, cal);
+    const uint64_t out = kernel_ps((u128)m_bytes * cV + (u128)y_bytes * c0, 0,
+                                   2u * (uint64_t)m * alpha * (alpha + m) * tile_channels_out * cA, cal);
+    return saturate((u128)in + con + out);
+}
+
+// Winograd F(2x2, 3x3) as one kernel: HBM sees x, y and U only.  A work item (32 tiles x 128 output channels)
+// is a serial loop over blocks of 32 input channels; a block costs the delivery of sixteen 128 x 32 weight tiles
+// from L2 to the SM or its sixty-four small MMAs, whichever is larger; the item's epilogue is not overlapped
+// (the sixteen accumulators fill tensor memory).
+uint64_t fused_cost(const LayerShape& s, const Calibration& cal)
+{
+    const uint64_t tiles = (uint64_t)s.N * ceil_div(s.OH, 2) * ceil_div(s.OW, 2);
+    const uint64_t sms = cal.c[7] > 0 ? (uint64_t)cal.c[7] : 148;
+    const uint64_t x_bytes = 4ull * s.N * s.Cin * s.H * s.W;
+    const uint64_t y_bytes = 4ull * s.N * s.Cout * s.OH * s.OW;
+    const uint64_t u_bytes = 16ull * s.Cout * s.Cin * 4;
+    const uint64_t co_blocks = ceil_div(s.Cout, 128);
+    const uint64_t rounds = ceil_div(ceil_div(tiles, 32) * co_blocks, sms);
+    const uint64_t k_blocks = ceil_div(s.Cin, 32);
+    const uint64_t deliver_ps = 16ull * 128 * 32 * 4 * (uint64_t)cal.c[10] / 1000000ull;
+    const uint64_t block_ps = deliver_ps > (uint64_t)cal.c[11] ? deliver_ps : (uint64_t)cal.c[11];
+    const u128 item_ps = (u128)k_blocks * block_ps + (uint64_t)cal.c[12];
+    const u128 serial_as = (u128)rounds * item_ps * 1000000u;
+    // x comes from HBM once; the other channel blocks find it in L2
+    return kernel_ps((u128)(x_bytes + y_bytes + u_bytes) * (uint64_t)cal.c[0] + (u128)(co_blocks - 1) * x_bytes * (uint64_t)cal.c[1],
+                     serial_as, 0, cal);
 }
 
 }  // namespace
+
+bool fused_shape_ok(const LayerShape& s)
+{
+    return s.k == 3 && s.stride == 1 && s.dil == 1 && s.groups == 1 && s.Cin % 8 == 0 && s.pad <= 2;
+}
+
+// Eq. 2, made comparable across tile sizes: a per-tile count, so multiplied by the number of tiles; its third
+// term (the output transform) with the output-channel factor it lacks as printed.
+uint64_t paper_multiplications(const LayerShape& s, int n)
+{
+    const uint64_t a = (uint64_t)(n + s.k - 1);
+    const u128 tiles = (u128)s.N * ceil_div(s.OH, n) * ceil_div(s.OW, n);
+    const u128 per_tile = (u128)2 * s.Cin * a * a * a + (u128)s.Cin * s.Cout * a * a + (u128)s.Cout * n * a * (2 * n + s.k - 1);
+    return saturate(tiles * per_tile);
+}
 
 void winograd_chunking(const LayerShape& s, int m, int operand, int passes, const Calibration& cal,
                        int* chunk_images, int* n_chunks, uint64_t* cost_ps)
@@ -415,7 +463,7 @@ void winograd_chunking(const LayerShape& s, int m, int operand, int passes, cons
     // option A: the largest chunk the cap allows (the whole batch if it fits)
     const uint64_t chunkA = N < n_cap ? N : ceil_div(N, ceil_div(N, n_cap));
     const uint64_t nA = ceil_div(N, chunkA);
-    const uint64_t costA = nA * winograd_chunk_cost(s, m, operand, passes, chunkA, n_fit >= chunkA, cal);
+    const uint64_t costA = saturate((u128)nA * winograd_chunk_cost(s, m, operand, passes, chunkA, n_fit >= chunkA, cal));
     uint64_t best_cost = costA;
     uint64_t best_chunk = chunkA, best_n = nA;
     // Cutting the batch further so that a chunk's V and M stay in L2 was measured on B200 and never paid:
@@ -444,14 +492,24 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
     for (int g = 0; g < 4; ++g)
         for (int i = 0; i < 3; ++i)
             cands[3 + g * 3 + i] = {MNN_ALGO_WINOGRAD, kM[i], g < 2 ? MNN_OPERAND_TF32 : MNN_OPERAND_BF16, (g & 1) ? 3 : 1};
-    cands[15] = {0, 0, 0, 0};
+    cands[15] = {MNN_ALGO_WINOGRAD, 2, MNN_OPERAND_TF32, 1};      // the fused kernel
+    {
+        static const int kN[4] = {1, 2, 4, 6};
+        int arg = 0;
+        for (int i = 0; i < 4; ++i) {
+            d->paper_mul[i] = paper_multiplications(s, kN[i]);
+            if (d->paper_mul[i] < d->paper_mul[arg]) arg = i;
+        }
+        d->paper_n_hat = kN[arg];
+    }
 
     int chunk_of[MNN_N_CANDIDATES] = {0}, nch_of[MNN_N_CANDIDATES] = {0}, pts_of[MNN_N_CANDIDATES] = {0};
     int lhs_of[MNN_N_CANDIDATES] = {0};
     long long ppm_of[MNN_N_CANDIDATES] = {0};
 
-    for (int i = 0; i < 15; ++i) {
+    for (int i = 0; i < MNN_N_CANDIDATES; ++i) {
         const Cand& c = cands[i];
+        if (o.fused == 2 && i != 15) continue;                     // the fused kernel or nothing
         if (o.force_algo != MNN_ALGO_AUTO && o.force_algo != c.algo) continue;
         if (c.algo == MNN_ALGO_DIRECT) {
             if (o.operand == MNN_OPERAND_FP32_REF || o.operand == MNN_OPERAND_AUTO || o.force_algo == MNN_ALGO_DIRECT)
@@ -479,6 +537,8 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
             continue;
         }
         // Winograd
+        const bool fused = i == 15;
+        if (fused && (o.fused == 1 || !fused_shape_ok(s) || cal.c[10] <= 0 || cal.c[11] <= 0)) continue;
         if (!wino_shape_ok || !winograd_supported(c.m, s.k)) continue;
         if (o.force_m != 0 && o.force_m != c.m) continue;
         long long ppm = 0;
@@ -490,12 +550,18 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
         pts_of[i] = pid;
         ppm_of[i] = ppm;
         uint64_t cost;
-        winograd_chunking(s, c.m, c.operand, c.passes, cal, &chunk_of[i], &nch_of[i], &cost);
+        if (fused) {
+            chunk_of[i] = s.N;
+            nch_of[i] = 1;
+            cost = fused_cost(s, cal);
+        } else {
+            winograd_chunking(s, c.m, c.operand, c.passes, cal, &chunk_of[i], &nch_of[i], &cost);
+        }
         d->cost_ps[i] = cost;
     }
 
     int best = -1;
-    for (int i = 0; i < 15; ++i)
+    for (int i = 0; i < MNN_N_CANDIDATES; ++i)
         if (d->cost_ps[i] != MNN_COST_INADMISSIBLE && (best < 0 || d->cost_ps[i] < d->cost_ps[best])) best = i;
 
     // A forced combination outside the candidate list (other m, fp32 checking contraction).
@@ -560,7 +626,8 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
         d->points_id = pts_of[best];
         d->chunk_images = chunk_of[best];
         d->n_chunks = nch_of[best];
-        if (o.chunk_images > 0) {
+        d->fused = best == 15 ? 1 : 0;
+        if (o.chunk_images > 0 && !d->fused) {
             d->chunk_images = o.chunk_images < s.N ? o.chunk_images : s.N;
             d->n_chunks = (s.N + d->chunk_images - 1) / d->chunk_images;
         }

@@ -21,6 +21,9 @@ struct Decision {
     int chunk_images = 0, n_chunks = 0;
     int chosen = -1;
     int gemm_lhs = 0;                  // MNN_GEMM_LHS_PATCHES or MNN_GEMM_LHS_X for the GEMM scheme, else 0
+    int fused = 0;                     // Winograd F(2x2,3x3) as the single fused kernel
+    int paper_n_hat = 0;               // Eq. 2's argmin over n in {1, 2, 4, 6} and the counts themselves
+    uint64_t paper_mul[4] = {0, 0, 0, 0};
     long long error_ppm = 0;
     uint64_t cost_ps[MNN_N_CANDIDATES];
 };
@@ -62,6 +65,9 @@ void winograd_chunking(const LayerShape& s, int m, int operand, int passes, cons
                        int* chunk_images, int* n_chunks, uint64_t* cost_ps);
 
 // Fills *d.  Returns MNN_OK or an mnn_status with *err set to a static reason.
+// True when the layer's shape admits the fused Winograd F(2x2, 3x3) kernel.
+bool fused_shape_ok(const LayerShape& s);
+
 int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& cal, Decision* d, const char** err);
 
 // True when the Winograd kernels exist for (m, k).
