@@ -237,7 +237,7 @@ def winograd_cost(L: Layer, m: int, operand: int, passes: int, c):
 # accumulators of a block of 128 output channels x 32 tiles in tensor memory.  HBM sees x, y and U only.
 # ---------------------------------------------------------------------------------------
 def fused_supported(L: Layer) -> bool:
-    return L.k == 3 and L.stride == 1 and L.dil == 1 and L.groups == 1 and L.Cin % 8 == 0 and L.pad <= 2
+    return L.k == 3 and L.stride == 1 and L.dil == 1 and L.groups == 1 and L.pad <= 2
 
 
 def fused_cost(L: Layer, c) -> int:

@@ -12,6 +12,7 @@
 #include "generator.h"
 #include "kernels.h"
 #include "planner.h"
+#include "wino_fused.h"
 
 using namespace mnnb;
 
@@ -101,8 +102,8 @@ void layout_workspace(mnn_conv_plan_t p)
         p->cin_pad = (int)align_up(s.Cin, 8);
         p->chunk_tiles = (long long)d.chunk_images * th * tw;
         p->m_row_stride = (int)align_up(p->chunk_tiles, 32);
-        p->u_bytes = align_up(a2 * s.Cout * p->cin_pad * eb, 2048);
         p->fused = d.fused != 0;
+        p->u_bytes = p->fused ? align_up(fused_wino_weight_bytes(s.Cout, s.Cin), 2048) : align_up(a2 * s.Cout * p->cin_pad * eb, 2048);
         p->v_bytes = p->fused ? 0 : align_up(a2 * p->chunk_tiles * p->cin_pad * eb, 2048);
         p->m_bytes = p->fused ? 0 : align_up(a2 * s.Cout * p->m_row_stride * 4, 1024);
         p->launches_per_run = p->fused ? 1 : 3 * d.n_chunks;
@@ -288,7 +289,7 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
 static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
 {
     const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
-    if (p->fused) return fused_wino_setup(&p->fw, p->s.Cout, p->cin_pad, u_hi(p), why);
+    if (p->fused) return fused_wino_setup(&p->fw, p->s.Cout, p->s.Cin, u_hi(p), why);
     if (p->gemm_x) return umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), why);
     return umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
                                v_lo(p), why);
@@ -382,7 +383,9 @@ static int do_weights(mnn_conv_plan_t p, const float* w, cudaStream_t st)
 {
     cudaError_t e;
     LaunchTimer lt(p, st, 0);
-    if (p->d.algo == MNN_ALGO_WINOGRAD)
+    if (p->fused)
+        e = launch_fused_wino_weights(w, u_hi(p), p->s.Cout, p->s.Cin, p->mats, st);
+    else if (p->d.algo == MNN_ALGO_WINOGRAD)
         e = launch_weight_transform(w, u_hi(p), u_lo(p), p->s.Cout, p->s.Cin, p->s.k, p->d.m, p->cin_pad, p->store_mode,
                                     p->mats, st);
     else

@@ -132,18 +132,6 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
 bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
                         long long plane_stride_elems, int box_rows);
 
-// Winograd F(2x2, 3x3) in one kernel (input transform, contraction and output transform fused; V and M never
-// reach global memory).  U is the transformed weight tensor [16][Cout][cin_pad] in TF32 (STORE_TF32).
-struct FusedWino {
-    CUtensorMap map_u;
-    int Cout = 0, cin_pad = 0, num_sms = 0, u_stages = 0, smem_bytes = 0;
-    bool ready = false;
-};
-bool fused_wino_applies(int k, int stride, int dil, int groups, int Cin, int pad, long long tiles);
-cudaError_t fused_wino_setup(FusedWino* fw, int Cout, int cin_pad, void* U, const char** why);
-cudaError_t launch_fused_wino(const FusedWino& fw, const float* x, const float* bias, float* y, const WinoGeom& g, int relu,
-                              const TransformMatrices& mats, int* status, cudaStream_t stream);
-
 // Direct ("sliding window") convolution, any stride / padding / dilation / groups.
 struct DirectGeom {
     int N, Cin, Cout, H, W, OH, OW, k, stride, pad, dil, groups, relu;

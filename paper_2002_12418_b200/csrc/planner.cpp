@@ -433,7 +433,7 @@ uint64_t fused_cost(const LayerShape& s, const Calibration& cal)
 
 bool fused_shape_ok(const LayerShape& s)
 {
-    return s.k == 3 && s.stride == 1 && s.dil == 1 && s.groups == 1 && s.Cin % 8 == 0 && s.pad <= 2;
+    return s.k == 3 && s.stride == 1 && s.dil == 1 && s.groups == 1 && s.pad <= 2;
 }
 
 // Eq. 2, made comparable across tile sizes: a per-tile count, so multiplied by the number of tiles; its third

@@ -30,7 +30,10 @@ def stage_work(info, N, Cin, Cout, H, W, k, groups):
     y_bytes = 4 * N * Cout * info.OH * info.OW
     b_el = (2 if info.operand == B.OPERAND_BF16 else 4) * (2 if info.passes == 3 else 1)
     out = {}
-    if info.algo == B.ALGO_WINOGRAD:
+    if info.algo == B.ALGO_WINOGRAD and info.fused:
+        T = N * (-(-info.OH // 2)) * (-(-info.OW // 2))
+        out["contract"] = (x_bytes + y_bytes + 4 * 16 * Cout * Cin, 2 * 16 * Cout * Cin * T)
+    elif info.algo == B.ALGO_WINOGRAD:
         a2 = info.alpha ** 2
         T = N * (-(-info.OH // info.m)) * (-(-info.OW // info.m))
         v, mm, u = b_el * a2 * Cin * T, 4 * a2 * Cout * T, b_el * a2 * Cout * Cin
@@ -71,6 +74,7 @@ def main():
     ap.add_argument("--stages", default="all", choices=sorted(STAGES))
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--flush", action="store_true", help="write 256 MB between repetitions")
+    ap.add_argument("--fused", type=int, default=0, help="0 planner, 1 never, 2 the single-kernel F(2x2,3x3) path")
     args = ap.parse_args()
 
     import torch
@@ -80,7 +84,7 @@ def main():
     pad = (args.k - 1) // 2 if args.pad < 0 else args.pad
     o = B.make_opts(groups=args.groups, relu=1, precision=B.PREC_TF32 if args.precision == "tf32" else B.PREC_BF16,
                     operand=OPERANDS[args.operand], passes=args.passes, force_algo=ALGOS[args.algo], force_m=args.m,
-                    chunk_images=args.chunk, gemm_lhs=LHS[args.lhs])
+                    chunk_images=args.chunk, gemm_lhs=LHS[args.lhs], fused=args.fused)
     r = B.ConvLayerRunner(args.N, Cin, Cout, args.H, args.H, args.k, args.stride, pad, 1, o)
     info = r.info
     g = torch.Generator(device="cpu").manual_seed(1)
@@ -118,7 +122,7 @@ def main():
     total_ms = sum(s["ms"] for s in stages.values())
     direct = 2 * args.N * Cout * (Cin // args.groups) * info.OH * info.OW * args.k * args.k
     print(json.dumps({"algo": B.ALGO_NAMES[info.algo], "m": info.m, "operand": B.OPERAND_NAMES[info.operand],
-                      "passes": info.passes, "gemm_lhs": info.gemm_lhs, "chunk_images": info.chunk_images, "n_chunks": info.n_chunks,
+                      "passes": info.passes, "gemm_lhs": info.gemm_lhs, "fused": info.fused, "chunk_images": info.chunk_images, "n_chunks": info.n_chunks,
                       "workspace_MB": round(info.workspace_bytes / 2 ** 20, 1), "device_status": status,
                       "stages": stages, "sum_ms": round(total_ms, 5),
                       "direct_equiv_TFLOPs": round(direct / total_ms / 1e9, 1) if total_ms > 0 else None}))

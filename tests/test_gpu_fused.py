@@ -78,7 +78,9 @@ def test_config1_batch32_sampled(torch):
     (3, 40, 136, 13, 9, 1),      # odd output sizes, two channel blocks with a ragged second one
     (2, 64, 72, 33, 20, 0),      # no padding, even OW
     (1, 16, 16, 6, 10, 2),       # pad 2: outputs larger than the input
-    (5, 32, 200, 5, 5, 1),       # more tile blocks than... a single partial block per image row
+    (5, 32, 200, 5, 5, 1),       # 3 x 3 tiles per image: blocks straddle images
+    (2, 3, 16, 12, 12, 1),       # three input channels (one partly filled K block)
+    (1, 21, 33, 9, 9, 1),        # odd channel counts on both sides
 ])
 def test_odd_shapes(torch, N, Cin, Cout, H, W_, pad):
     layer = W.ConvLayer("t", N, Cin, Cout, H, W_, 3, 1, pad, relu=True, x_dist="normal", w_dist="kaiming", seed=N * 7 + Cin)
@@ -118,7 +120,6 @@ def test_repeatable(torch):
 
 def test_where_it_does_not_apply(torch):
     for args, kw in (((1, 16, 16, 8, 8, 3, 2, 1, 1), {}),          # stride 2
-                     ((1, 12, 16, 8, 8, 3, 1, 1, 1), {}),          # Cin not a multiple of 8
                      ((1, 16, 16, 8, 8, 5, 1, 2, 1), {}),          # 5x5
                      ((1, 16, 16, 8, 8, 3, 1, 1, 1), {"operand": B.OPERAND_BF16})):
         with pytest.raises(B.MnnError):
