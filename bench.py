@@ -1,13 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the convolution hot path on B200.
 
-A step = one forward pass of every layer of the workload (ResNet-18-style 3x3
-stride-1 layers at batch 32: weights already transformed, inputs resident in HBM)
+A step = one forward pass of every layer of the workload (default: the large-batch
+Winograd layers, batch 64: weights already transformed, inputs resident in HBM)
 through mnn_conv_run.  Prints ONE JSON line: direct-convolution-equivalent TFLOP/s,
-ms per step, the roofline position of the dominant kernel, the end-to-end figure with
-host buffers, and the CPU oracle timed beside it.
+ms per step, the roofline position of every stage and of the dominant kernel, a second
+block for the ResNet-18-style batch-32 layers, the end-to-end figure with host buffers,
+and the CPU oracle timed beside it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload config1_b32]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload config4_b64]
+
+With --gpus N > 1 on a plain command line the benchmark starts the N local ranks itself;
+under a launcher that already set RANK / WORLD_SIZE (torchrun) it is one of the ranks.
 """
 from __future__ import annotations
 
@@ -27,11 +31,13 @@ if ROOT not in sys.path:
 METRIC = "conv TFLOP/s (direct-conv-equivalent)"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch (mean over the four layers of one step) from one ncu
-# capture of this file's default workload (profiles/bench_config1_b32_launch_list.md gives the command).  Valid
-# for config1_b32 / tf32 and the kernels as captured; set an entry to None when its kernel changes.
-NCU_DRAM_BYTES_PER_LAUNCH = {"config1_b32/tf32": {"input": 40.30e6, "contraction": 45.51e6, "output": 15.49e6}}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from stored ncu captures of
+# this file's workloads (profiles/ holds the summaries and their commands); not measured by this run.  An entry is
+# used only while the plans of the run are the plans of the capture.
+NCU_DRAM_TRAFFIC = {}
 
+# nominal dense tensor rates relative to BF16 (2.25 PFLOP/s): TF32 1.1 PFLOP/s
+TF32_OVER_BF16 = 1.1 / 2.25
 
 def workload_layers(name: str):
     from paper_2002_12418_b200 import workloads as W
@@ -148,24 +154,59 @@ def time_oracle_sample(layers, images=4, min_seconds=0.0):
     return total_flops, total_s, oc.threads()
 
 
+def time_oracle_outputs(layers, outputs_per_layer):
+    """The oracle on `outputs_per_layer` seeded output coordinates of the first image pair of every layer (for
+    workloads whose single images are already too large for the time budget of a step)."""
+    from oracle import direct_conv as oc
+    from paper_2002_12418_b200 import workloads as W
+    import numpy as np
+    total_flops, total_s = 0, 0.0
+    for layer in layers:
+        part = layer.with_batch(min(2, layer.N))
+        x, w, b = W.make_inputs(part)
+        n_out = part.N * part.Cout * part.OH * part.OW
+        idx = np.random.Generator(np.random.PCG64(part.seed + 1)).integers(0, n_out, size=min(outputs_per_layer, n_out))
+        t0 = time.perf_counter()
+        y = oc.direct_conv_at(x, w, b, idx, part.stride, part.pad, part.dilation, part.groups, part.relu)
+        total_s += time.perf_counter() - t0
+        total_flops += 2 * (part.Cin // part.groups) * part.k * part.k * len(idx)
+        assert np.isfinite(y).all()
+    return total_flops, total_s, oc.threads()
+
+
 def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the workload per step: up to four whole images of every
+    layer, fewer when K steps of that would not end within about three minutes, and for the largest layers a seeded
+    set of output coordinates instead of whole images."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     layers = workload_layers(args.workload)
     from oracle import direct_conv as oc
     oc.build()
-    for _ in range(min(args.warmup, 1)):
-        time_oracle_sample(layers[:1])
+    # rate estimate from one small run (also the warm-up)
+    f0, s0, cores = time_oracle_sample(layers[-1:], images=1)
+    rate = f0 / max(s0, 1e-6)
+    budget_flops = rate * 180.0 / max(args.steps, 1)                 # per step
+    per_image = sum(l.direct_flops // l.N for l in layers)
+    images = int(min(4, budget_flops // per_image))
     flops, secs = 0, 0.0
-    cores = 1
-    for _ in range(args.steps):
-        f, s, cores = time_oracle_sample(layers)
-        flops += f
-        secs += s
+    if images >= 1:
+        for _ in range(args.steps):
+            f, s, cores = time_oracle_sample(layers, images=images)
+            flops += f
+            secs += s
+        what = "first %d image(s) of each of the %d layers per step" % (images, len(layers))
+    else:
+        per_output = sum(2 * (l.Cin // l.groups) * l.k * l.k for l in layers) / len(layers)
+        n_out = max(1024, int(budget_flops / len(layers) / per_output))
+        for _ in range(args.steps):
+            f, s, cores = time_oracle_outputs(layers, n_out)
+            flops += f
+            secs += s
+        what = "%d seeded output coordinates of each of the %d layers per step" % (n_out, len(layers))
     value = flops / secs / 1e12
-    sample = "first 4 images of each of the %d layers per step (%.3f GFLOP direct per step), fp64 nested loops" % (
-        len(layers), flops / args.steps / 1e9)
+    sample = "%s (%.3f GFLOP direct per step), fp64 nested loops" % (what, flops / args.steps / 1e9)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
@@ -186,7 +227,10 @@ def stage_work(layer, info):
     y_bytes = 4 * N * Cout * info.OH * info.OW
     b_el = (2 if info.operand == B.OPERAND_BF16 else 4) * (2 if info.passes == 3 else 1)
     out = {}
-    if info.algo == B.ALGO_WINOGRAD:
+    if info.algo == B.ALGO_WINOGRAD and info.fused:
+        T = N * (-(-info.OH // 2)) * (-(-info.OW // 2))
+        out["contraction"] = {"bytes": x_bytes + y_bytes + 4 * 16 * Cout * Cin, "flops": 2 * 16 * Cout * Cin * T}
+    elif info.algo == B.ALGO_WINOGRAD:
         a2 = info.alpha ** 2
         th, tw = -(-info.OH // info.m), -(-info.OW // info.m)
         T = N * th * tw
@@ -209,31 +253,180 @@ def stage_work(layer, info):
     return out
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="config1_b32")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--precision", default="tf32", choices=["tf32", "bf16"])
-    ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
-                    help="how a timed step is issued: one CUDA-graph replay of the step's launches (captured "
-                         "once from the same C-ABI calls), or the calls themselves on the stream")
-    ap.add_argument("--calibration", default="measure", choices=["measure", "builtin"],
-                    help="measure: run mnn_calibrate on this GPU before planning (default); builtin: plan from the "
-                         "library's frozen B200 record (use under a profiler, which slows the calibration launches)")
-    args = ap.parse_args()
-    if args.impl == "reference":
-        run_reference(args)
-        return
-
-    import numpy as np
+def build_state(layers, prec, dev, rank, world):
     import torch
     from paper_2002_12418_b200 import binding as B
     from paper_2002_12418_b200 import replicas as R
     from paper_2002_12418_b200 import workloads as W
+    state = []
+    for layer in layers:
+        # every rank works on its own batch of the same shape (weak scaling; images are independent)
+        lay = layer if world == 1 else layer.with_batch(layer.N, seed_offset=R.rank_seed_offset(rank))
+        x, w, b = W.make_inputs(lay)
+        o = B.make_opts(groups=lay.groups, relu=lay.relu, precision=prec)
+        r = B.ConvLayerRunner(lay.N, lay.Cin, lay.Cout, lay.H, lay.W, lay.k, lay.stride, lay.pad, lay.dilation, o,
+                              device=str(dev))
+        xd = torch.from_numpy(x).to(dev)
+        wd = torch.from_numpy(w).to(dev)
+        bd = torch.from_numpy(b).to(dev) if b is not None else None
+        yd = torch.empty((lay.N, lay.Cout, r.info.OH, r.info.OW), dtype=torch.float32, device=dev)
+        r.prepare(wd)
+        state.append({"layer": lay, "runner": r, "x": xd, "w": wd, "b": bd, "y": yd, "x_host": x})
+    return state
+
+
+def check_status(state, where):
+    for s in state:
+        code = s["runner"].device_status()
+        if code != 0:
+            raise SystemExit("bench: a kernel of %s reported a bounded wait that ran out (code %d) %s: the "
+                             "timing is void" % (s["layer"].name, code, where))
+
+
+def arithmetic_label(state):
+    from paper_2002_12418_b200 import binding as B
+    kinds = []
+    for s in state:
+        info = s["runner"].info
+        if info.algo == B.ALGO_DIRECT:
+            k = "f32"
+        else:
+            k = "%sx%d" % (B.OPERAND_NAMES[info.operand], info.passes)
+        if k not in kinds:
+            kinds.append(k)
+    return "+".join(kinds)
+
+
+def time_workload(state, steps, warmup, launch, flush, dev, dist, barrier, sample_clocks):
+    """K timed steps (L2 flushed before each, CUDA events on the launching stream), then the same steps again with
+    events around every launch for the per-stage figures.  Returns a dict."""
+    import torch
+    from paper_2002_12418_b200 import binding as B
+    from paper_2002_12418_b200 import replicas as R
+    stream = torch.cuda.current_stream(dev)
+    world = dist.get_world_size() if dist is not None else 1
+
+    def one_step():
+        for s in state:
+            s["runner"].run(s["x"], s["w"], s["b"], s["y"])
+
+    for _ in range(max(warmup, 3)):
+        flush.zero_()
+        one_step()
+    barrier()
+    check_status(state, "during warm-up")
+    y_first = [s["y"].clone() for s in state]
+
+    # The step's launches captured once into a CUDA graph: the same C-ABI calls, recorded instead of run.
+    timed_step = one_step
+    if launch == "graph":
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(step_graph):
+            one_step()
+        timed_step = step_graph.replay
+        for _ in range(3):
+            flush.zero_()
+            timed_step()
+        barrier()
+
+    sampler = None
+    if sample_clocks:
+        sampler = ClockSampler(dev.index or 0)
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t_wall0 = time.time()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for k in range(steps):
+        flush.zero_()
+        ev[k][0].record(stream)
+        timed_step()
+        ev[k][1].record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler is not None else None
+    check_status(state, "in the timed region")
+    for s, y0 in zip(state, y_first):
+        if not torch.equal(s["y"], y0):
+            raise SystemExit("bench: %s gave a different result in the timed region than in warm-up" % s["layer"].name)
+    total_ms = float(sum(a.elapsed_time(b) for a, b in ev))
+    total_ms = R.max_over_ranks(dist, total_ms, dev)
+    flops_step = sum(s["layer"].direct_flops for s in state)
+    value = R.whole_job_throughput(flops_step, steps, world, total_ms)
+    launches = sum(s["runner"].info.launches_per_run for s in state) * steps
+
+    # ---- per-kernel durations (events around every launch), same steps again ----
+    stage_names = ["weight", "input", "contraction", "output"]
+    stage_ms = {n: 0.0 for n in stage_names}
+    stage_n = {n: 0 for n in stage_names}
+    stage_bytes = {n: 0 for n in stage_names}
+    tensor_flops, tensor_roof_s = 0.0, 0.0          # executed MMA flops and the time the measured peak would need
+    peaks = measured_peaks()
+    per_layer = []
+    prof_steps = min(steps, 200)
+    for s in state:
+        B.mnn_conv_profile(s["runner"].plan, True)
+    for k in range(prof_steps):
+        flush.zero_()
+        one_step()
+        for s in state:
+            ms, n = B.mnn_conv_profile_read(s["runner"].plan)
+            info = s["runner"].info
+            work = stage_work(s["layer"], info)
+            for i, nm in enumerate(stage_names):
+                stage_ms[nm] += ms[i]
+                stage_n[nm] += n[i]
+                if n[i] and nm in work:
+                    stage_bytes[nm] += work[nm]["bytes"]
+            if info.algo != B.ALGO_DIRECT and n[2]:
+                fl = work["contraction"]["flops"]
+                peak = peaks["bf16_tflops"] * (1.0 if info.operand == B.OPERAND_BF16 else TF32_OVER_BF16)
+                tensor_flops += fl
+                tensor_roof_s += fl / (peak * 1e12)
+            if k == prof_steps - 1:
+                per_layer.append({"name": s["layer"].name, "algo": B.ALGO_NAMES[info.algo], "m": info.m,
+                                  "operand": B.OPERAND_NAMES[info.operand], "passes": info.passes, "fused": info.fused,
+                                  "chunk_images": info.chunk_images, "stage_ms_last_step": [round(v, 4) for v in ms]})
+    for s in state:
+        B.mnn_conv_profile(s["runner"].plan, False)
+    torch.cuda.synchronize(dev)
+    check_status(state, "in the per-launch timing pass")
+
+    stages = {}
+    for nm in stage_names:
+        if stage_n[nm] == 0:
+            continue
+        sec = stage_ms[nm] * 1e-3
+        gbs = stage_bytes[nm] / sec / 1e9
+        stages[nm] = {"ms_per_step": stage_ms[nm] / prof_steps, "launches_per_step": stage_n[nm] // prof_steps,
+                      "avg_launch_us": stage_ms[nm] / stage_n[nm] * 1e3,
+                      "algorithmic_GBps": gbs, "frac_of_hbm": gbs / peaks["hbm_gbs"]}
+    if tensor_flops > 0 and "contraction" in stages:
+        sec = stage_ms["contraction"] * 1e-3
+        stages["contraction"]["tensor_TFLOPs"] = tensor_flops / sec / 1e12
+        stages["contraction"]["frac_of_tensor_peak"] = tensor_roof_s / sec
+    dominant = max(stages, key=lambda n: stages[n]["ms_per_step"])
+    d = stages[dominant]
+    if dominant == "contraction" and d.get("frac_of_tensor_peak", 0.0) >= d["frac_of_hbm"]:
+        # the dense contraction against the measured tensor peak of each layer's operand format (burst figure: the
+        # kernel is timed alone by its own events); TF32 = measured BF16 x the nominal ratio 1.1 / 2.25
+        roofline = {"kernel": dominant, "bound": "tensor", "achieved": d["tensor_TFLOPs"],
+                    "peak": d["tensor_TFLOPs"] / d["frac_of_tensor_peak"], "unit": "TFLOP/s",
+                    "frac": d["frac_of_tensor_peak"]}
+    else:
+        roofline = {"kernel": dominant, "bound": "hbm", "achieved": d["algorithmic_GBps"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": d["frac_of_hbm"]}
+    roofline.update({"peak_source": peaks["source"] + " (MEASURED_PEAKS.json)" if peaks["source"] == "measured" else "fallback",
+                     "avg_launch_us": d["avg_launch_us"], "launches": stage_n[dominant], "traffic": None,
+                     "stages": stages})
+    return {"value": value, "ms_per_step": total_ms / steps, "launches": launches, "flops_step": flops_step,
+            "roofline": roofline, "plans": per_layer, "clocks": clocks, "arithmetic": arithmetic_label(state)}
+
+
+def gpu_rank_main(args):
+    import torch
+    from paper_2002_12418_b200 import binding as B
+    from paper_2002_12418_b200 import replicas as R
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -253,7 +446,6 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    layers = workload_layers(args.workload)
     prec = B.PREC_TF32 if args.precision == "tf32" else B.PREC_BF16
     # pre-inference: the planner's cost constants are measured once on this GPU, before any plan is made
     if args.calibration == "measure":
@@ -261,114 +453,17 @@ def main():
         torch.cuda.synchronize(dev)
     else:
         calibration = B.mnn_get_calibration()
-    # every rank works on its own batch of the same shape (weak scaling; images are independent)
-    state = []
-    for i, layer in enumerate(layers):
-        lay = layer if world == 1 else layer.with_batch(layer.N, seed_offset=R.rank_seed_offset(rank))
-        x, w, b = W.make_inputs(lay)
-        o = B.make_opts(groups=lay.groups, relu=lay.relu, precision=prec)
-        r = B.ConvLayerRunner(lay.N, lay.Cin, lay.Cout, lay.H, lay.W, lay.k, lay.stride, lay.pad, lay.dilation, o,
-                              device=str(dev))
-        xd = torch.from_numpy(x).to(dev)
-        wd = torch.from_numpy(w).to(dev)
-        bd = torch.from_numpy(b).to(dev) if b is not None else None
-        yd = torch.empty((lay.N, lay.Cout, r.info.OH, r.info.OW), dtype=torch.float32, device=dev)
-        r.prepare(wd)
-        state.append({"layer": lay, "runner": r, "x": xd, "w": wd, "b": bd, "y": yd, "x_host": x})
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream(dev)
 
-    def one_step():
-        for s in state:
-            s["runner"].run(s["x"], s["w"], s["b"], s["y"])
-
-    for _ in range(max(args.warmup, 3)):
-        flush.zero_()
-        one_step()
-    barrier()
-    for s in state:
-        assert s["runner"].device_status() == 0, "a kernel reported a bounded wait that ran out"
-
-    # The step's launches captured once into a CUDA graph: the same C-ABI calls, recorded instead of run.
-    # Replaying it issues the same kernels with the same arguments without the per-launch host work.
-    timed_step = one_step
-    if args.launch == "graph":
-        step_graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(step_graph):
-            one_step()
-        timed_step = step_graph.replay
-        for _ in range(3):
-            flush.zero_()
-            timed_step()
-        barrier()
-
-    # ---- timed region: K steps, L2 flushed before each, device time by CUDA events ----
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    time.sleep(0.3)
-    barrier()
-    t_wall0 = time.time()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for k in range(args.steps):
-        flush.zero_()
-        ev[k][0].record(stream)
-        timed_step()
-        ev[k][1].record(stream)
-    barrier()
-    t_wall1 = time.time()
-    step_ms = [a.elapsed_time(b) for a, b in ev]
-    clocks = sampler.stop(t_wall0, t_wall1)
-    total_ms = float(sum(step_ms))
-    total_ms = R.max_over_ranks(dist, total_ms, dev)
-    flops_step = sum(s["layer"].direct_flops for s in state)
-    value = R.whole_job_throughput(flops_step, args.steps, world, total_ms)
-    launches = sum(s["runner"].info.launches_per_run for s in state) * args.steps
-
-    # ---- per-kernel durations (events around every launch), same steps again ----
-    stage_names = ["weight", "input", "contraction", "output"]
-    stage_ms = {n: 0.0 for n in stage_names}
-    stage_n = {n: 0 for n in stage_names}
-    stage_bytes = {n: 0 for n in stage_names}
-    stage_flops = {n: 0 for n in stage_names}
-    per_layer = []
-    for s in state:
-        B.mnn_conv_profile(s["runner"].plan, True)
-    for k in range(args.steps):
-        flush.zero_()
-        one_step()
-        for s in state:
-            ms, n = B.mnn_conv_profile_read(s["runner"].plan)
-            work = stage_work(s["layer"], s["runner"].info)
-            for i, nm in enumerate(stage_names):
-                stage_ms[nm] += ms[i]
-                stage_n[nm] += n[i]
-                if n[i] and nm in work:
-                    stage_bytes[nm] += work[nm]["bytes"]
-                    stage_flops[nm] += work[nm]["flops"]
-            if k == args.steps - 1:
-                info = s["runner"].info
-                per_layer.append({"name": s["layer"].name, "algo": B.ALGO_NAMES[info.algo], "m": info.m,
-                                  "operand": B.OPERAND_NAMES[info.operand], "passes": info.passes,
-                                  "chunk_images": info.chunk_images, "stage_ms_last_step": [round(v, 4) for v in ms]})
-    for s in state:
-        B.mnn_conv_profile(s["runner"].plan, False)
-    torch.cuda.synchronize(dev)
-    peaks = measured_peaks()
-    dominant = max(stage_names, key=lambda n: stage_ms[n])
-    dom_launches = max(stage_n[dominant], 1)
-    dom_ms = stage_ms[dominant] / dom_launches
-    dom_bytes = stage_bytes[dominant] / dom_launches
-    achieved_gbs = dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    roofline = {"kernel": dominant, "bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved_gbs / peaks["hbm_gbs"],
-                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get("%s/%s" % (args.workload, args.precision), {}).get(dominant),
-                "algorithmic_bytes_per_launch": dom_bytes, "peak_source": peaks["source"],
-                "avg_launch_us": dom_ms * 1e3, "launches": stage_n[dominant],
-                "stage_ms_per_step": {n: stage_ms[n] / args.steps for n in stage_names},
-                "stage_gbs": {n: (stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 if stage_ms[n] > 0 else None)
-                              for n in stage_names},
-                "contraction_tflops": (stage_flops["contraction"] / (stage_ms["contraction"] * 1e-3) / 1e12
-                                       if stage_ms["contraction"] > 0 else None)}
+    layers = workload_layers(args.workload)
+    state = build_state(layers, prec, dev, rank, world)
+    main_res = time_workload(state, args.steps, args.warmup, args.launch, flush, dev, dist, barrier, True)
+    key = "%s/%s" % (args.workload, args.precision)
+    stored = NCU_DRAM_TRAFFIC.get(key)
+    if stored and stored.get("plans") == [(p["algo"], p["m"], p["operand"], p["passes"]) for p in main_res["plans"]]:
+        main_res["roofline"]["traffic"] = stored.get(main_res["roofline"]["kernel"])
+        main_res["roofline"]["traffic_source"] = stored["source"]
 
     # ---- end to end through the public call with HOST buffers ----
     h2d = sum(s["x_host"].nbytes for s in state)
@@ -417,9 +512,23 @@ def main():
     e2e_join()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = R.max_over_ranks(dist, e2e_ms, dev)
-    e2e_value = R.whole_job_throughput(flops_step, e2e_steps, world, e2e_ms)
+    check_status(state, "in the end-to-end leg")
+    e2e_ms = R.max_over_ranks(dist, e0.elapsed_time(e1), dev)
+    e2e_value = R.whole_job_throughput(main_res["flops_step"], e2e_steps, world, e2e_ms)
+    for s in state:
+        s["runner"].close()
+    del state
+
+    # ---- second workload, reported beside the headline (never as the headline) ----
+    secondary = None
+    if args.secondary and args.secondary != args.workload:
+        st2 = build_state(workload_layers(args.secondary), prec, dev, rank, world)
+        r2 = time_workload(st2, max(20, min(args.steps, 400)), args.warmup, args.launch, flush, dev, dist, barrier, False)
+        secondary = {"workload": args.secondary, "value": r2["value"], "unit": UNIT, "ms_per_step": r2["ms_per_step"],
+                     "dtype": r2["arithmetic"], "gpu_launches": r2["launches"], "roofline": r2["roofline"],
+                     "plans": r2["plans"]}
+        for s in st2:
+            s["runner"].close()
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -429,21 +538,69 @@ def main():
                                   "all), fp64 nested loops" % (len(layers), secs, f / 1e9)}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if prec == B.PREC_TF32 else "bf16",
-                "data": "synthetic",
+        line = {"metric": METRIC, "value": main_res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": main_res["ms_per_step"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": main_res["arithmetic"], "data": "synthetic",
                 "config": {"workload": args.workload, "layers": len(layers), "batch_per_gpu": layers[0].N,
                            "l2": "flushed before every step (256 MB write)", "weights": "pre-transformed",
                            "launch": "CUDA graph replay per step" if args.launch == "graph" else "C-ABI calls on the stream",
-                           "accuracy_class": args.precision, "planner_calibration": calibration[:9], "calibration_source": args.calibration, "plans": per_layer},
-                "clocks": clocks, "roofline": roofline,
+                           "accuracy_class": args.precision, "planner_calibration": calibration[:13],
+                           "calibration_source": args.calibration, "plans": main_res["plans"]},
+                "clocks": main_res["clocks"], "roofline": main_res["roofline"],
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms / e2e_steps},
-                "gpu_launches": launches, "cpu_baseline": cpu_baseline}
+                "gpu_launches": main_res["launches"], "device_status": 0, "secondary": secondary,
+                "cpu_baseline": cpu_baseline}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def _spawned_rank(rank, world, port, argv):
+    from paper_2002_12418_b200 import replicas as R
+    os.environ.update(R.rank_environment(rank, world, port))
+    sys.argv = argv
+    gpu_rank_main(parse_args())
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config4_b64")
+    ap.add_argument("--secondary", default="config1_b32", help="a second workload reported beside the headline ('' = none)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--precision", default="tf32", choices=["tf32", "bf16"])
+    ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
+                    help="how a timed step is issued: one CUDA-graph replay of the step's launches (captured "
+                         "once from the same C-ABI calls), or the calls themselves on the stream")
+    ap.add_argument("--calibration", default="measure", choices=["measure", "builtin"],
+                    help="measure: run mnn_calibrate on this GPU before planning (default); builtin: plan from the "
+                         "library's frozen B200 record (use under a profiler, which slows the calibration launches)")
+    return ap.parse_args()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    from paper_2002_12418_b200 import replicas as R
+    how = R.launch_plan(args.gpus, os.environ)
+    if how == "spawn":
+        # a plain command line asked for N GPUs: start the N local ranks here (NCCL only for the barrier and the
+        # max-over-ranks time; no data-path collective)
+        import socket
+        import torch.multiprocessing as mp
+        s = socket.socket()
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+        s.close()
+        mp.spawn(_spawned_rank, args=(args.gpus, port, list(sys.argv)), nprocs=args.gpus, join=True)
+        return
+    gpu_rank_main(args)
 
 
 if __name__ == "__main__":

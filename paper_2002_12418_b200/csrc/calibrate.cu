@@ -13,6 +13,7 @@
 #include "generator.h"
 #include "kernels.h"
 #include "planner.h"
+#include "wino_fused.h"
 
 using namespace mnnb;
 
@@ -235,6 +236,57 @@ extern "C" int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CO
             const long long measured = to_ll(t * 1e15 / flops);
             // the run is partly memory-bound, so this is an upper bound on the ALU cost
             if (measured < cal.c[4]) cal.c[4] = measured;
+        }
+    }
+
+    // fused F(2x2,3x3) kernel: one work item (32 tiles x 128 output channels) with 32 and with 256 input channels;
+    // the difference is seven blocks of 32 input channels, the rest of the short run is launch and epilogue
+    {
+        WinogradMatrices wm;
+        if (generate_winograd(2, 3, 2, &wm)) {
+            TransformMatrices mats;
+            std::memset(&mats, 0, sizeof(mats));
+            std::memcpy(mats.At, wm.At32.data(), wm.At32.size() * sizeof(float));
+            std::memcpy(mats.G, wm.G32.data(), wm.G32.size() * sizeof(float));
+            std::memcpy(mats.Bt, wm.Bt32.data(), wm.Bt32.size() * sizeof(float));
+            double t_of[2] = {0.0, 0.0};
+            bool ok = true;
+            for (int v = 0; v < 2 && ok; ++v) {
+                const int cin = v == 0 ? 32 : 256, cout = 128;
+                WinoGeom g;
+                g.images = 2; g.Cin = cin; g.Cout = cout; g.H = 8; g.W = 8; g.OH = 8; g.OW = 8; g.k = 3; g.pad = 1;
+                g.m = 2; g.alpha = 4; g.th = 4; g.tw = 4; g.cin_pad = cin;
+                g.tiles = 32; g.v_plane = 0; g.m_row_stride = 0;
+                int* status = reinterpret_cast<int*>(buf);
+                float* x = reinterpret_cast<float*>(buf + 1024);
+                float* w = x + (size_t)2 * 256 * 64;
+                float* y = w + (size_t)128 * 256 * 9;
+                char* U = buf + (8 << 20);
+                cudaMemsetAsync(buf, 0, 1024, st);
+                FusedWino fw;
+                const char* why = "";
+                if (fused_wino_setup(&fw, cout, cin, U, &why) != cudaSuccess ||
+                    launch_fused_wino_weights(w, U, cout, cin, mats, st) != cudaSuccess) {
+                    ok = false;
+                    break;
+                }
+                for (int i = 0; i < 3; ++i) launch_fused_wino(fw, x, nullptr, y, g, 0, mats, status, st);
+                tm.start();
+                const int reps = 20;
+                for (int i = 0; i < reps; ++i) launch_fused_wino(fw, x, nullptr, y, g, 0, mats, status, st);
+                t_of[v] = tm.stop() / reps;
+                int code = 0;
+                cudaMemcpy(&code, status, sizeof(int), cudaMemcpyDeviceToHost);
+                if (code != 0 || !(t_of[v] > 0.0)) ok = false;
+            }
+            if (ok && t_of[1] > t_of[0]) {
+                const double block_ms = (t_of[1] - t_of[0]) / 7.0;
+                cal.c[11] = to_ll(block_ms * 1e9);
+                cal.c[10] = to_ll(block_ms * 1e15 / (16.0 * 128 * 32 * 4));
+                double epi_ms = t_of[0] - block_ms - (double)cal.c[5] * 1e-9;
+                if (epi_ms < block_ms * 0.25) epi_ms = block_ms * 0.25;
+                cal.c[12] = to_ll(epi_ms * 1e9);
+            }
         }
     }
 

@@ -53,9 +53,9 @@ Calibration default_calibration()
     c.c[7] = 148;         // SMs
     c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
     c.c[9] = 60000;       // as per flop of the direct kernel for Cin <= 4 (~17 TFLOP/s)
-    c.c[10] = 8000;       // as per byte of U delivered from L2 to one SM by the fused kernel (~125 GB/s per SM)
-    c.c[11] = 1300000;    // ps of tensor work per 32-channel block of a fused work item (64 MMAs of 128 x 32 x 8)
-    c.c[12] = 1500000;    // ps of epilogue per fused work item
+    c.c[10] = 23000000;   // as per byte of U delivered to one SM by the fused kernel's weight stream (~43 GB/s per SM)
+    c.c[11] = 6000000;    // ps per 32-channel block of a fused work item (64 MMAs of 128 x 32 x 8 at ~90 ns each)
+    c.c[12] = 4300000;    // ps of epilogue per fused work item
     return c;
 }
 

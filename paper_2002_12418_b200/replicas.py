@@ -22,3 +22,18 @@ def max_over_ranks(dist, value: float, device=None) -> float:
 def whole_job_throughput(flops_per_rank_step: float, steps: int, world: int, slowest_ms: float) -> float:
     """Aggregate TFLOP/s of `world` replicas that each did `steps` steps in at most `slowest_ms`."""
     return world * flops_per_rank_step * steps / (slowest_ms * 1e-3) / 1e12
+
+
+def launch_plan(gpus: int, env) -> str:
+    """How `bench.py --gpus N` gets its N ranks: "single" (N = 1), "env" (a launcher such as torchrun
+    already started one process per rank: WORLD_SIZE is set), or "spawn" (N > 1 asked for on a plain
+    command line: the benchmark starts the N local ranks itself)."""
+    if "WORLD_SIZE" in env and int(env["WORLD_SIZE"]) >= 1 and "RANK" in env:
+        return "env"
+    return "single" if gpus <= 1 else "spawn"
+
+
+def rank_environment(rank: int, world: int, port: int) -> dict:
+    """Rendezvous variables of one locally spawned rank."""
+    return {"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world), "MASTER_ADDR": "127.0.0.1",
+            "MASTER_PORT": str(port)}

@@ -60,3 +60,12 @@ def test_single_rank_needs_no_process_group():
     assert R.max_over_ranks(None, 3.5) == 3.5
     assert R.rank_seed_offset(0) == 0 and R.rank_seed_offset(3) == 30000
     assert np.isclose(R.whole_job_throughput(1e12, 10, 1, 1000.0), 10.0)
+
+
+def test_launch_plan_spawns_ranks_only_on_a_plain_command_line():
+    assert R.launch_plan(1, {}) == "single"
+    assert R.launch_plan(8, {}) == "spawn"
+    assert R.launch_plan(8, {"WORLD_SIZE": "8", "RANK": "3"}) == "env"
+    assert R.launch_plan(1, {"WORLD_SIZE": "1", "RANK": "0"}) == "env"
+    env = R.rank_environment(2, 4, 29512)
+    assert env == {"RANK": "2", "LOCAL_RANK": "2", "WORLD_SIZE": "4", "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": "29512"}
