@@ -94,7 +94,14 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
  *              transform fused; the transformed tensors V and M never reach device memory):
  *              0 = the planner weighs it against the other candidates, 1 = never,
  *              2 = this kernel or fail.  It applies to 3x3 stride-1 undilated ungrouped layers with
- *              Cin a multiple of 8 and pad <= 2, accuracy class permitting single-pass TF32 at m = 2.
+ *              pad <= 2, accuracy class permitting single-pass TF32 at m = 2.
+ *   strassen   1 = run a 1x1 stride-1 unpadded layer's matrix product through ONE recursion level of
+ *              Strassen's algorithm (Section 3.3.2): seven half-size products in one batched contraction,
+ *              the additions folded into one pass before and one after it.  Needs even N, Cin and Cout.
+ *              Unless operand/passes are given, the operands are BF16 hi + lo (3 passes) under the TF32
+ *              accuracy class (the sums and differences of products lose about a factor three of
+ *              accuracy) and single-pass TF32 under the BF16 class.  0 = plain product (the planner
+ *              never chooses Strassen by itself: on this GPU it loses at every size a layer produces).
  */
 typedef struct {
     int groups;
@@ -108,7 +115,8 @@ typedef struct {
     int chunk_images;
     int gemm_lhs;
     int fused;
-    int reserved[5];
+    int strassen;
+    int reserved[4];
 } mnn_conv_opts;
 
 /*
@@ -144,6 +152,8 @@ typedef struct {
     int fused;                       /* 1 when the plan is the single fused Winograd kernel (no V, no M) */
     int paper_n_hat;
     unsigned long long paper_mul[4];
+    int strassen;                    /* 1 when the plan runs one Strassen level (alpha = 1, seven products) */
+    int reserved0;
 } mnn_conv_info;
 
 /* Plan one layer with groups = 1, relu = 1, accuracy class TF32, everything else
@@ -225,6 +235,7 @@ MNN_API void mnn_conv_destroy(mnn_conv_plan_t plan);
  *     batch, or a smaller tile size, to fit.
  *   - the first call on each device looks up the array's device address (with
  *     that device current); make that first call outside any stream capture.
+ *     The current device must be the device of `stream` in every call.
  *   - every call on a device uses the same array, which keeps the previous
  *     call's contents; the call clears the one word that must start at zero.
  *     Two calls that overlap on the GPU (different streams, or different
@@ -248,6 +259,12 @@ MNN_API int mnn_winograd_matrices(int m, int k, int points_id, float* At, float*
  * simulation with rounded operands; the planner's accuracy gate.  m = 1 with
  * points_id = 0 gives the figure of the GEMM scheme (no transforms).  < 0 on error. */
 MNN_API long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int passes);
+
+/* The paper's stopping rule for the Strassen recursion (Eq. 9) for a product [n x k] times [k x m]:
+ * 1 when m n k - 7 (m/2)(n/2)(k/2) > 4 (m/2)(k/2) + 4 (n/2)(k/2) + 7 (m/2)(n/2), i.e. when the multiplications
+ * saved outnumber the additions added, counting both alike; else 0.  Reported for comparison: it weighs a
+ * multiplication like an addition, which does not hold where the multiplications run on tensor cores. */
+MNN_API int mnn_strassen_rule(long long m, long long n, long long k);
 
 /* Cost-model constants (Eq. 5's FLOPS and t_schedule, re-stated for this GPU).
  * consts[0] attoseconds per HBM byte          consts[1] attoseconds per L2-resident byte

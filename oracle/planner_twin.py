@@ -223,8 +223,8 @@ def winograd_cost(L: Layer, m: int, operand: int, passes: int, c):
     c_vm = c[1] if fits_l2 >= chunk else c[0]
     # ALU work of the transforms: 2 alpha^3 multiply-adds per (tile, channel) on the input side (the first term
     # of Eq. 2), m alpha (alpha + m) on the output side (its third term); from alpha = 8 a lane holds one channel
-    # instead of a pair (x2), from alpha = 10 the tile no longer fits the register file (x4)
-    crowding = 4 if alpha >= 10 else (2 if alpha >= 8 else 1)
+    # instead of a pair (x2), from alpha = 10 the tile no longer fits the register file (x4; x8 at alpha = 12)
+    crowding = 8 if alpha >= 12 else (4 if alpha >= 10 else (2 if alpha >= 8 else 1))
     t_in = kernel_ps(c, mem_as=x * c[0] + v * c_vm, alu_as=crowding * 4 * alpha * a2 * n * tiles_img * L.Cin * c[4])
     t_con = kernel_ps(c, mem_as=(v + mm) * c_vm + u * c[0],
                       tensor_as=2 * a2 * L.Cout * Cp * n * tiles_img * passes * _tensor_rate(c, operand))
@@ -460,3 +460,14 @@ def accuracy_ppm(m: int, k: int, points_id: int, operand: int, passes: int, gene
                 ref += np.einsum("oc,tcab->toab", w[:, :, i, j], x[:, :, i:i + m, j:j + m])
     rel = math.sqrt(float(((got - ref) ** 2).sum()) / float((ref ** 2).sum()))
     return int(math.ceil(rel * 1e6))
+
+
+# ---------------------------------------------------------------------------------------
+# Strassen's stopping rule (Eq. 9) for [n x k] x [k x m]: recurse while the multiplications saved outnumber
+# the additions added, both counted alike.
+# ---------------------------------------------------------------------------------------
+def strassen_rule(m: int, n: int, k: int) -> bool:
+    if min(m, n, k) < 2:
+        return False
+    mh, nh, kh = m // 2, n // 2, k // 2
+    return m * n * k - 7 * mh * nh * kh > 4 * mh * kh + 4 * nh * kh + 7 * mh * nh

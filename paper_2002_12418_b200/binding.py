@@ -27,7 +27,7 @@ OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "
 
 EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_query", "mnn_conv_set_workspace",
             "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
-            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_calibrate",
+            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_strassen_rule", "mnn_calibrate",
             "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error",
             "mnn_net_plan", "mnn_net_query", "mnn_net_set_workspace", "mnn_net_prepare", "mnn_net_run",
             "mnn_net_device_status", "mnn_net_destroy"]
@@ -38,7 +38,7 @@ class ConvOpts(ctypes.Structure):
     _fields_ = [("groups", ctypes.c_int), ("relu", ctypes.c_int), ("precision", ctypes.c_int),
                 ("operand", ctypes.c_int), ("passes", ctypes.c_int), ("force_algo", ctypes.c_int),
                 ("force_m", ctypes.c_int), ("points_id", ctypes.c_int), ("chunk_images", ctypes.c_int),
-                ("gemm_lhs", ctypes.c_int), ("fused", ctypes.c_int), ("reserved", ctypes.c_int * 5)]
+                ("gemm_lhs", ctypes.c_int), ("fused", ctypes.c_int), ("strassen", ctypes.c_int), ("reserved", ctypes.c_int * 4)]
 
 
 class ConvInfo(ctypes.Structure):
@@ -54,7 +54,8 @@ class ConvInfo(ctypes.Structure):
                 ("predicted_error_ppm", ctypes.c_longlong),
                 ("chosen_candidate", ctypes.c_int), ("gemm_lhs", ctypes.c_int),
                 ("cost_ps", ctypes.c_ulonglong * N_CANDIDATES),
-                ("fused", ctypes.c_int), ("paper_n_hat", ctypes.c_int), ("paper_mul", ctypes.c_ulonglong * 4)]
+                ("fused", ctypes.c_int), ("paper_n_hat", ctypes.c_int), ("paper_mul", ctypes.c_ulonglong * 4),
+                ("strassen", ctypes.c_int), ("reserved0", ctypes.c_int)]
 
 
 class LayerDesc(ctypes.Structure):
@@ -119,6 +120,8 @@ def lib():
         L.mnn_winograd_matrices.restype = i
         L.mnn_accuracy_ppm.argtypes = [i] * 5
         L.mnn_accuracy_ppm.restype = ll
+        L.mnn_strassen_rule.argtypes = [ll, ll, ll]
+        L.mnn_strassen_rule.restype = i
         L.mnn_calibrate.argtypes = [i, p, ctypes.POINTER(ll)]
         L.mnn_calibrate.restype = i
         L.mnn_set_calibration.argtypes = [ctypes.POINTER(ll)]
@@ -155,12 +158,13 @@ def _check(rc: int) -> None:
 
 
 def make_opts(groups=1, relu=0, precision=PREC_TF32, operand=0, passes=0, force_algo=0, force_m=0, points_id=0,
-              chunk_images=0, gemm_lhs=0, fused=0) -> ConvOpts:
+              chunk_images=0, gemm_lhs=0, fused=0, strassen=0) -> ConvOpts:
     o = ConvOpts()
     o.groups, o.relu, o.precision, o.operand, o.passes = groups, int(bool(relu)), precision, operand, passes
     o.force_algo, o.force_m, o.points_id, o.chunk_images = force_algo, force_m, points_id, chunk_images
     o.gemm_lhs = gemm_lhs
     o.fused = fused
+    o.strassen = strassen
     return o
 
 
@@ -247,6 +251,10 @@ def mnn_accuracy_ppm(m, k, points_id, operand, passes) -> int:
     if v < 0:
         raise MnnError(MNN_EINVAL, mnn_last_error())
     return int(v)
+
+
+def mnn_strassen_rule(m: int, n: int, k: int) -> int:
+    return int(lib().mnn_strassen_rule(m, n, k))
 
 
 def mnn_calibrate(device: int, stream: int) -> list[int]:

@@ -12,6 +12,7 @@
 #include "generator.h"
 #include "kernels.h"
 #include "planner.h"
+#include "strassen.h"
 #include "wino_fused.h"
 
 using namespace mnnb;
@@ -56,6 +57,7 @@ struct mnn_conv_plan_s {
     long long ws_bytes = 0;
     const float* prepared_w = nullptr;
     UmmaContract uc;
+    bool strassen = false;           // GEMM scheme through one Strassen level: seven half-size products
     bool fused = false;              // Winograd F(2x2,3x3) as the single fused kernel: the workspace holds U only
     FusedWino fw;
     // optional per-launch timing
@@ -107,6 +109,15 @@ void layout_workspace(mnn_conv_plan_t p)
         p->v_bytes = p->fused ? 0 : align_up(a2 * p->chunk_tiles * p->cin_pad * eb, 2048);
         p->m_bytes = p->fused ? 0 : align_up(a2 * s.Cout * p->m_row_stride * 4, 1024);
         p->launches_per_run = p->fused ? 1 : 3 * d.n_chunks;
+    } else if (p->strassen) {
+        const long long Mh = s.Cout / 2;
+        p->cin_pad = (int)align_up(s.Cin / 2, 8);
+        p->chunk_tiles = (long long)(s.N / 2) * s.OH * s.OW;
+        p->m_row_stride = (int)align_up(p->chunk_tiles, 32);
+        p->u_bytes = align_up(7 * Mh * p->cin_pad * eb, 2048);
+        p->v_bytes = align_up(7 * p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->m_bytes = align_up(7 * Mh * p->m_row_stride * 4, 1024);
+        p->launches_per_run = 3;
     } else {
         p->cin_pad = (int)align_up((long long)s.Cin * s.k * s.k, 8);
         p->chunk_tiles = (long long)s.N * s.OH * s.OW;
@@ -186,7 +197,7 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
     }
     if (o.operand < 0 || o.operand > MNN_OPERAND_FP32_REF || !(o.passes == 0 || o.passes == 1 || o.passes == 3) ||
         o.force_algo < 0 || o.force_algo > MNN_ALGO_DIRECT || o.points_id < 0 || o.points_id > MNN_POINTS_MIXED ||
-        o.force_m < 0 || o.chunk_images < 0 || o.gemm_lhs < 0 || o.gemm_lhs > MNN_GEMM_LHS_X || o.fused < 0 || o.fused > 2) {
+        o.force_m < 0 || o.chunk_images < 0 || o.gemm_lhs < 0 || o.gemm_lhs > MNN_GEMM_LHS_X || o.fused < 0 || o.fused > 2 || o.strassen < 0 || o.strassen > 1) {
         fail(MNN_EINVAL, "an option is outside its range");
         return nullptr;
     }
@@ -207,6 +218,22 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
         fail(MNN_EUNSUPPORTED, "tensor too large");
         return nullptr;
     }
+    if (o.strassen) {
+        if (!strassen_applies(N, Cin, Cout, k, stride, pad, dilation, o.groups) || o.force_algo == MNN_ALGO_WINOGRAD ||
+            o.force_algo == MNN_ALGO_DIRECT || o.operand == MNN_OPERAND_FP32_REF || o.gemm_lhs == MNN_GEMM_LHS_X) {
+            fail(MNN_EUNSUPPORTED, "Strassen needs a 1x1 stride-1 unpadded ungrouped layer with even N, Cin and Cout on the GEMM scheme");
+            return nullptr;
+        }
+        // the sums and differences of the seven products lose about a factor three of accuracy
+        o.force_algo = MNN_ALGO_GEMM;
+        o.gemm_lhs = MNN_GEMM_LHS_PATCHES;
+        if (o.operand == MNN_OPERAND_AUTO) {
+            o.operand = o.precision == MNN_PREC_TF32 ? MNN_OPERAND_BF16 : MNN_OPERAND_TF32;
+            o.passes = o.precision == MNN_PREC_TF32 ? 3 : 1;
+        } else if (o.passes == 0) {
+            o.passes = 1;
+        }
+    }
     mnn_conv_plan_t p = new (std::nothrow) mnn_conv_plan_s();
     if (!p) {
         fail(MNN_EINVAL, "out of host memory");
@@ -214,12 +241,21 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
     }
     p->s = s;
     p->o = o;
+    p->strassen = o.strassen != 0;
     const char* why = "";
-    int rc = plan_layer(s, o, current_calibration(), &p->d, &why);
+    mnn_conv_opts o_plan = o;
+    if (p->strassen) o_plan.passes = 1;      // the candidate list holds single-pass GEMMs; the pass count is set below
+    int rc = plan_layer(s, o_plan, current_calibration(), &p->d, &why);
     if (rc != MNN_OK) {
         fail(rc, why);
         delete p;
         return nullptr;
+    }
+    if (p->strassen) {
+        p->d.passes = o.passes;
+        p->d.chosen = -1;
+        p->d.gemm_lhs = MNN_GEMM_LHS_PATCHES;
+        p->d.error_ppm = accuracy_ppm(1, 1, 0, p->d.operand, p->d.passes);
     }
     if (p->d.algo == MNN_ALGO_WINOGRAD) {
         WinogradMatrices wm;
@@ -280,6 +316,8 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     info->gemm_lhs = p->d.algo == MNN_ALGO_GEMM ? p->d.gemm_lhs : 0;
     for (int i = 0; i < MNN_N_CANDIDATES; ++i) info->cost_ps[i] = p->d.cost_ps[i];
     info->fused = p->fused ? 1 : 0;
+    info->strassen = p->strassen ? 1 : 0;
+    if (p->strassen) info->predicted_error_ppm = 3 * p->d.error_ppm;
     info->paper_n_hat = p->d.paper_n_hat;
     for (int i = 0; i < 4; ++i) info->paper_mul[i] = p->d.paper_mul[i];
     return MNN_OK;
@@ -290,6 +328,9 @@ static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
 {
     const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
     if (p->fused) return fused_wino_setup(&p->fw, p->s.Cout, p->s.Cin, u_hi(p), why);
+    if (p->strassen)
+        return umma_contract_setup(&p->uc, p->store_mode, 7, p->s.Cout / 2, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
+                                   v_lo(p), why);
     if (p->gemm_x) return umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), why);
     return umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
                                v_lo(p), why);
@@ -365,7 +406,7 @@ static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, con
     const bool need_x = direct || (!one_kernel && (mask & MNN_STAGE_INPUT)) || (one_kernel && (mask & MNN_STAGE_CONTRACT));
     const bool need_w = direct || (mask & MNN_STAGE_WEIGHT);
     const bool need_y = direct || (!p->fused && (mask & MNN_STAGE_OUTPUT)) ||
-                        ((p->d.algo == MNN_ALGO_GEMM || p->fused) && (mask & MNN_STAGE_CONTRACT));
+                        (((p->d.algo == MNN_ALGO_GEMM && !p->strassen) || p->fused) && (mask & MNN_STAGE_CONTRACT));
     if ((need_x && !x) || (need_w && !w) || (need_y && !y)) return fail(MNN_EINVAL, "NULL tensor pointer");
     if ((x && !aligned16(x)) || (w && !aligned16(w)) || (y && !aligned16(y)))
         return fail(MNN_EALIGN, "x, w and y must be 16-byte aligned");
@@ -379,11 +420,23 @@ static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, con
     return MNN_OK;
 }
 
+static StrassenGeom strassen_geom(mnn_conv_plan_t p)
+{
+    StrassenGeom g;
+    g.N = p->s.N; g.Cin = p->s.Cin; g.Cout = p->s.Cout; g.HW = p->s.H * p->s.W;
+    g.k_pad = p->cin_pad;
+    g.t_half = p->chunk_tiles;
+    g.m_row_stride = p->m_row_stride;
+    return g;
+}
+
 static int do_weights(mnn_conv_plan_t p, const float* w, cudaStream_t st)
 {
     cudaError_t e;
     LaunchTimer lt(p, st, 0);
-    if (p->fused)
+    if (p->strassen)
+        e = launch_strassen_weights(w, u_hi(p), u_lo(p), strassen_geom(p), p->store_mode, st);
+    else if (p->fused)
         e = launch_fused_wino_weights(w, u_hi(p), p->s.Cout, p->s.Cin, p->mats, st);
     else if (p->d.algo == MNN_ALGO_WINOGRAD)
         e = launch_weight_transform(w, u_hi(p), u_lo(p), p->s.Cout, p->s.Cin, p->s.k, p->d.m, p->cin_pad, p->store_mode,
@@ -435,6 +488,27 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
     }
     const bool reference = d.operand == MNN_OPERAND_FP32_REF;
 
+    if (p->strassen) {
+        const StrassenGeom g = strassen_geom(p);
+        if (reference) return fail(MNN_EUNSUPPORTED, "Strassen runs on the tensor-core contraction only");
+        if (mask & MNN_STAGE_INPUT) {
+            LaunchTimer lt(p, st, 1);
+            e = launch_strassen_input(x, v_hi(p), v_lo(p), g, p->store_mode, st);
+            if (e != cudaSuccess) return fail_cuda(e, "Strassen operand pass");
+        }
+        if (mask & MNN_STAGE_CONTRACT) {
+            ContractEpilogue epi = {0, m_buf(p), p->m_row_stride, nullptr, nullptr, 0, 1};
+            LaunchTimer lt(p, st, 2);
+            e = launch_contract_umma(p->uc, g.t_half, epi, status_word(p), st);
+            if (e != cudaSuccess) return fail_cuda(e, "Strassen products");
+        }
+        if (mask & MNN_STAGE_OUTPUT) {
+            LaunchTimer lt(p, st, 3);
+            e = launch_strassen_output(m_buf(p), bias, y, g, s.relu, st);
+            if (e != cudaSuccess) return fail_cuda(e, "Strassen result pass");
+        }
+        return MNN_OK;
+    }
     if (d.algo == MNN_ALGO_GEMM) {
         const long long T = (long long)s.N * s.OH * s.OW;
         if ((mask & MNN_STAGE_INPUT) && !p->gemm_x) {
@@ -598,6 +672,15 @@ long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int passes)
     long long v = accuracy_ppm(m, k, points_id, operand, passes);
     if (v < 0) fail(MNN_EINVAL, "invalid (m, k, points_id, operand, passes)");
     return v;
+}
+
+int mnn_strassen_rule(long long m, long long n, long long k)
+{
+    if (m < 2 || n < 2 || k < 2) return 0;
+    const __int128 mh = m / 2, nh = n / 2, kh = k / 2;
+    const __int128 saved = (__int128)m * n * k - 7 * mh * nh * kh;
+    const __int128 added = 4 * mh * kh + 4 * nh * kh + 7 * mh * nh;
+    return saved > added ? 1 : 0;
 }
 
 int mnn_set_calibration(const long long consts[MNN_N_CONSTS])

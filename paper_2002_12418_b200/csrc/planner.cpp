@@ -395,9 +395,10 @@ uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes
     const uint64_t cV = (uint64_t)(resident ? cal.c[1] : cal.c[0]);
     const uint64_t c0 = (uint64_t)cal.c[0], cA = (uint64_t)cal.c[4];
     // from alpha = 8 on a lane of the input transform holds one channel instead of a packed pair (twice the ALU
-    // time); from alpha = 10 on the tile no longer fits the register file (measured about twice that again)
+    // time); from alpha = 10 on the tile no longer fits the register file (measured about twice that again, and
+    // twice again at alpha = 12)
     const u128 tile_channels_in = (u128)n * tiles_img * (uint64_t)s.Cin, tile_channels_out = (u128)n * tiles_img * (uint64_t)s.Cout;
-    const u128 in_alu = (alpha >= 10 ? 4u : (alpha >= 8 ? 2u : 1u)) * 4u * alpha * a2 * tile_channels_in * cA;
+    const u128 in_alu = (alpha >= 12 ? 8u : (alpha >= 10 ? 4u : (alpha >= 8 ? 2u : 1u))) * 4u * alpha * a2 * tile_channels_in * cA;
     const uint64_t in = kernel_ps((u128)x_bytes * c0 + (u128)v_bytes * cV, 0, in_alu, cal);
     const uint64_t con = kernel_ps((u128)(v_bytes + m_bytes) * cV + (u128)u_bytes * c0,
                                    2u * a2 * Cp * tile_channels_out * (uint64_t)passes * tensor_as(operand, cal), 0, cal);

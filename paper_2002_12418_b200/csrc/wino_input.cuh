@@ -275,7 +275,6 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
         for (unsigned li = 0; li < n_local; ++li) {
             if (round > 0 && !ptx::mbar_wait_relaxed(ptx::smem_u32(&empty_bar[b]), (round - 1) & 1u, abortp)) {
                 if (!*abortp && status) atomicCAS(status, 0, kErrInputLoaderWait | (int)(min(li, 0xFFFFu) << 8) | (int)((blockIdx.x & 0x7Fu) << 24));
-                if (status && lane == 0) { atomicCAS(status + 1, 0, (int)(0x40000000u | li | (b << 16) | (blockIdx.x << 20))); }
                 *abortp = 1;
                 break;
             }

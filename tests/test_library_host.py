@@ -28,7 +28,7 @@ def test_struct_layouts_match_the_header():
     # sizes follow from the field lists in the header (ints 4 bytes, long long 8)
     import ctypes
     assert ctypes.sizeof(B.ConvOpts) == 16 * 4
-    assert ctypes.sizeof(B.ConvInfo) == 16 * 4 + 9 * 8 + 2 * 4 + 16 * 8 + 2 * 4 + 4 * 8
+    assert ctypes.sizeof(B.ConvInfo) == 16 * 4 + 9 * 8 + 2 * 4 + 16 * 8 + 2 * 4 + 4 * 8 + 2 * 4
 
 
 @pytest.mark.parametrize("m,k", [(m, k) for m in (1, 2, 3, 4, 6, 8) for k in (1, 2, 3, 5, 7)])

@@ -4,14 +4,17 @@ Some users of the library are given their tensors by a host application and may 
 create device memory themselves (a plug-in under another framework's memory budget, a
 real-time loop that must not make calls which can block on the driver).  For them the
 library carries a fixed built-in workspace.  This file checks, through the C ABI, that a
-layer run on that built-in workspace gives the same result as the same plan run on a
-caller-provided workspace — twice in a row with different layers, because the built-in
-array is shared and keeps the previous call's contents — and that a plan too large for
-it is refused.  It is collected last so that a failure here cannot hide other tests.
+layer run on that built-in workspace gives bit for bit the result of the same plan run on
+a caller-provided workspace (the kernels are deterministic, so anything but equality would
+be a fault) and meets the accuracy class against the fp64 oracle — several calls in a row
+with different layers, because the built-in array is shared and keeps the previous call's
+contents, among them a layer whose channel padding must be zero-filled on the dirty array
+— and that a plan too large for it is refused.  It is collected last so that a failure here cannot hide other tests.
 """
 import numpy as np
 import pytest
 
+from oracle import direct_conv as oc
 from paper_2002_12418_b200 import binding as B
 from paper_2002_12418_b200 import workloads as W
 from tests.util import assert_close, to_dev
@@ -34,6 +37,9 @@ def _both_ways(torch, layer, opts):
     torch.cuda.synchronize()
     ref, got = y_ref.cpu().numpy(), y_new.cpu().numpy()
     r.close()
+    assert np.array_equal(got, ref), "the static run differs from the run on a caller's workspace"
+    want = oc.direct_conv(x, w, b, layer.stride, layer.pad, layer.dilation, layer.groups, layer.relu)
+    assert_close(got, want, B.PREC_TF32, layer.name + " against the oracle")
     return got, ref
 
 
@@ -55,6 +61,13 @@ def test_static_workspace_run_matches_workspace_run_twice():
     c = W.ConvLayer("c", 2, 32, 48, 15, 15, 3, 2, 1, relu=True, seed=903)
     got, ref = _both_ways(torch, c, B.make_opts(relu=1, force_algo=B.ALGO_GEMM, operand=B.OPERAND_TF32))
     assert_close(got, ref, B.PREC_TF32, "third call")
+    # a channel count that is not a multiple of 8: the padding columns of U and V must be written as zeros
+    # over whatever the larger layers above left in the array
+    d = W.ConvLayer("d", 2, 20, 40, 11, 11, 3, 1, 1, relu=True, seed=904)
+    _both_ways(torch, d, B.make_opts(relu=1, force_algo=B.ALGO_WINOGRAD, force_m=4, operand=B.OPERAND_BF16, passes=3))
+    # the single-kernel Winograd path keeps only its packed weights in the array
+    e = W.ConvLayer("e", 2, 24, 136, 12, 12, 3, 1, 1, relu=True, seed=905)
+    _both_ways(torch, e, B.make_opts(relu=1, fused=B.FUSED_ONLY))
 
 
 def test_static_workspace_rejects_plans_that_do_not_fit():
