@@ -151,3 +151,45 @@ int oracle_direct_conv_f64_at(const float* x, const float* w, const float* bias,
     }
     return 0;
 }
+
+/*
+ * Rectangular kernels (the paper's Section 4.2 names the 1 x 7 and 7 x 1 convolutions of Inception-v3):
+ * the same definition with its own kernel height and width and its own padding per axis, stride 1,
+ * no dilation, one group:
+ *
+ *   y[n,co,oh,ow] = act( bias[co] + sum_ci sum_{a<kh} sum_{b<kw}
+ *                        w[co,ci,a,b] * xpad[n, ci, oh - pad_h + a, ow - pad_w + b] )
+ *   OH = H + 2 pad_h - kh + 1,  OW = W + 2 pad_w - kw + 1;   w is [Cout][Cin][kh][kw].
+ */
+int oracle_direct_conv_rect_f64(const float* x, const float* w, const float* bias, double* y,
+                                int N, int Cin, int Cout, int H, int W, int kh, int kw,
+                                int pad_h, int pad_w, int relu)
+{
+    if (N < 0 || Cin <= 0 || Cout <= 0 || H <= 0 || W <= 0 || kh <= 0 || kw <= 0 || pad_h < 0 || pad_w < 0)
+        return -1;
+    const int OH = H + 2 * pad_h - kh + 1, OW = W + 2 * pad_w - kw + 1;
+    if (OH <= 0 || OW <= 0) return -1;
+    const long long planes = (long long)N * Cout;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long long p = 0; p < planes; ++p) {
+        const int n = (int)(p / Cout), co = (int)(p % Cout);
+        for (int oh = 0; oh < OH; ++oh)
+            for (int ow = 0; ow < OW; ++ow) {
+                double acc = bias ? (double)bias[co] : 0.0;
+                for (int ci = 0; ci < Cin; ++ci)
+                    for (int a = 0; a < kh; ++a) {
+                        const int ih = oh - pad_h + a;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int b = 0; b < kw; ++b) {
+                            const int iw = ow - pad_w + b;
+                            if (iw < 0 || iw >= W) continue;
+                            acc += (double)w[(((size_t)co * Cin + ci) * kh + a) * kw + b] *
+                                   (double)x[(((size_t)n * Cin + ci) * H + ih) * W + iw];
+                        }
+                    }
+                if (relu && acc < 0.0) acc = 0.0;
+                y[((size_t)p * OH + oh) * OW + ow] = acc;
+            }
+    }
+    return 0;
+}

@@ -43,6 +43,8 @@ def _load():
         lib.oracle_direct_conv_f64_images.restype = i
         lib.oracle_direct_conv_f64_at.argtypes = [p, p, p, p, ll, p] + [i] * 11
         lib.oracle_direct_conv_f64_at.restype = i
+        lib.oracle_direct_conv_rect_f64.argtypes = [p, p, p, p] + [i] * 10
+        lib.oracle_direct_conv_rect_f64.restype = i
         _lib = lib
     return _lib
 
@@ -113,3 +115,26 @@ def direct_conv_at(x, w, bias, flat_indices, stride=1, pad=0, dil=1, groups=1, r
     if rc != 0:
         raise ValueError("oracle_direct_conv_f64_at rejected its arguments")
     return out
+
+
+def direct_conv_rect(x, w, bias=None, pad_h=0, pad_w=0, relu=False) -> np.ndarray:
+    """Rectangular kernel w [Cout,Cin,kh,kw], stride 1, its own padding per axis; fp64 [N,Cout,OH,OW]."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    if x.ndim != 4 or w.ndim != 4 or w.shape[1] != x.shape[1]:
+        raise ValueError("x must be [N,Cin,H,W], w [Cout,Cin,kh,kw]")
+    N, Cin, H, W = x.shape
+    Cout, _, kh, kw = w.shape
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        if bias.shape != (Cout,):
+            raise ValueError("bias must be [Cout]")
+    OH, OW = H + 2 * pad_h - kh + 1, W + 2 * pad_w - kw + 1
+    if OH <= 0 or OW <= 0:
+        raise ValueError("the kernel does not fit the padded input")
+    y = np.empty((N, Cout, OH, OW), dtype=np.float64)
+    rc = _load().oracle_direct_conv_rect_f64(_ptr(x), _ptr(w), _ptr(bias), _ptr(y), N, Cin, Cout, H, W, kh, kw,
+                                             pad_h, pad_w, int(bool(relu)))
+    if rc != 0:
+        raise ValueError("oracle_direct_conv_rect_f64 rejected its arguments")
+    return y

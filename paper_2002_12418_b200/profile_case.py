@@ -40,6 +40,12 @@ def stage_work(info, N, Cin, Cout, H, W, k, groups):
         out["input"] = (x_bytes + v, 0)
         out["contract"] = (v + mm + u * info.n_chunks, 2 * a2 * Cout * Cin * T * info.passes)
         out["output"] = (mm + y_bytes, 0)
+    elif info.algo == B.ALGO_GEMM and info.strassen:
+        T, Kh, Mh = N * info.OH * info.OW // 2, Cin // 2, Cout // 2
+        v, mm = b_el * 7 * T * Kh, 4 * 7 * Mh * T
+        out["input"] = (x_bytes + v, 0)
+        out["contract"] = (v + mm + b_el * 7 * Mh * Kh, 2 * 7 * Mh * Kh * T * info.passes)
+        out["output"] = (mm + y_bytes, 0)
     elif info.algo == B.ALGO_GEMM:
         K, T = Cin * k * k, N * info.OH * info.OW
         v = b_el * T * K
@@ -74,6 +80,7 @@ def main():
     ap.add_argument("--stages", default="all", choices=sorted(STAGES))
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--flush", action="store_true", help="write 256 MB between repetitions")
+    ap.add_argument("--strassen", type=int, default=0, help="1: one Strassen level on a 1x1 layer's product")
     ap.add_argument("--fused", type=int, default=0, help="0 planner, 1 never, 2 the single-kernel F(2x2,3x3) path")
     args = ap.parse_args()
 
@@ -84,7 +91,7 @@ def main():
     pad = (args.k - 1) // 2 if args.pad < 0 else args.pad
     o = B.make_opts(groups=args.groups, relu=1, precision=B.PREC_TF32 if args.precision == "tf32" else B.PREC_BF16,
                     operand=OPERANDS[args.operand], passes=args.passes, force_algo=ALGOS[args.algo], force_m=args.m,
-                    chunk_images=args.chunk, gemm_lhs=LHS[args.lhs], fused=args.fused)
+                    chunk_images=args.chunk, gemm_lhs=LHS[args.lhs], fused=args.fused, strassen=args.strassen)
     r = B.ConvLayerRunner(args.N, Cin, Cout, args.H, args.H, args.k, args.stride, pad, 1, o)
     info = r.info
     g = torch.Generator(device="cpu").manual_seed(1)
@@ -122,7 +129,7 @@ def main():
     total_ms = sum(s["ms"] for s in stages.values())
     direct = 2 * args.N * Cout * (Cin // args.groups) * info.OH * info.OW * args.k * args.k
     print(json.dumps({"algo": B.ALGO_NAMES[info.algo], "m": info.m, "operand": B.OPERAND_NAMES[info.operand],
-                      "passes": info.passes, "gemm_lhs": info.gemm_lhs, "fused": info.fused, "chunk_images": info.chunk_images, "n_chunks": info.n_chunks,
+                      "passes": info.passes, "gemm_lhs": info.gemm_lhs, "fused": info.fused, "strassen": info.strassen, "chunk_images": info.chunk_images, "n_chunks": info.n_chunks,
                       "workspace_MB": round(info.workspace_bytes / 2 ** 20, 1), "device_status": status,
                       "stages": stages, "sum_ms": round(total_ms, 5),
                       "direct_equiv_TFLOPs": round(direct / total_ms / 1e9, 1) if total_ms > 0 else None}))

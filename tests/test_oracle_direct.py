@@ -169,3 +169,64 @@ def test_rejects_bad_arguments():
         oc.direct_conv(x, w, None, 1, 0, 1, 2, False)       # 3 channels, 2 groups
     with pytest.raises(ValueError):
         oc.direct_conv(x, w, None, 0, 0, 1, 1, False)       # stride 0
+
+
+# ---------------------------------------------------------------------------
+# Rectangular kernels (Section 4.2: the 1 x 7 / 7 x 1 convolutions of Inception-v3).
+# ---------------------------------------------------------------------------
+def test_rect_hand_worked_cases():
+    import json
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "hand_rect_cases.json")
+    for case in json.load(open(path))["cases"]:
+        x = np.array(case["x"], dtype=np.float32)
+        w = np.array(case["w"], dtype=np.float32)
+        b = np.array(case["bias"], dtype=np.float32)
+        y = oc.direct_conv_rect(x, w, b, case["pad_h"], case["pad_w"], case["relu"])
+        assert np.array_equal(y, np.array(case["y"], dtype=np.float64)), case["name"]
+
+
+def _rect_other_order(x, w, b, ph, pw, relu):
+    """A second evaluation: one shifted, zero-padded copy of x per kernel tap, accumulated tap by tap."""
+    N, Cin, H, W = x.shape
+    Cout, _, kh, kw = w.shape
+    OH, OW = H + 2 * ph - kh + 1, W + 2 * pw - kw + 1
+    xp = np.zeros((N, Cin, H + 2 * ph, W + 2 * pw))
+    xp[:, :, ph:ph + H, pw:pw + W] = x
+    y = np.zeros((N, Cout, OH, OW))
+    for a in range(kh):
+        for c in range(kw):
+            y += np.einsum("oc,nchw->nohw", w[:, :, a, c].astype(np.float64), xp[:, :, a:a + OH, c:c + OW])
+    y += b.astype(np.float64)[None, :, None, None]
+    return np.maximum(y, 0) if relu else y
+
+
+@pytest.mark.parametrize("kh,kw,ph,pw", [(1, 3, 0, 1), (3, 1, 1, 0), (1, 7, 0, 3), (7, 1, 3, 0), (1, 5, 1, 0), (2, 3, 1, 2),
+                                         (3, 3, 1, 1), (1, 1, 0, 0)])
+def test_rect_against_a_second_evaluation_order(kh, kw, ph, pw):
+    rng = np.random.default_rng(kh * 10 + kw)
+    x = rng.standard_normal((2, 3, 6, 9)).astype(np.float32)
+    w = rng.standard_normal((4, 3, kh, kw)).astype(np.float32)
+    b = rng.standard_normal(4).astype(np.float32)
+    for relu in (False, True):
+        got = oc.direct_conv_rect(x, w, b, ph, pw, relu)
+        assert np.allclose(got, _rect_other_order(x, w, b, ph, pw, relu), rtol=0, atol=1e-12)
+
+
+def test_rect_reduces_to_the_square_definition_and_transposes():
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((2, 3, 7, 8)).astype(np.float32)
+    w = rng.standard_normal((5, 3, 3, 3)).astype(np.float32)
+    b = rng.standard_normal(5).astype(np.float32)
+    assert np.array_equal(oc.direct_conv_rect(x, w, b, 1, 1, True), oc.direct_conv(x, w, b, 1, 1, 1, 1, True))
+    # a 1 x k kernel on x equals the k x 1 kernel on the transposed image, transposed back
+    w17 = rng.standard_normal((5, 3, 1, 7)).astype(np.float32)
+    a = oc.direct_conv_rect(x, w17, b, 0, 3)
+    t = oc.direct_conv_rect(x.transpose(0, 1, 3, 2), w17.transpose(0, 1, 3, 2), b, 3, 0)
+    assert np.array_equal(a, t.transpose(0, 1, 3, 2))
+    # an off-centre delta tap shifts the image (catches a flipped kernel)
+    d = np.zeros((1, 1, 1, 3), dtype=np.float32)
+    d[0, 0, 0, 2] = 1
+    img = rng.standard_normal((1, 1, 2, 6)).astype(np.float32)
+    y = oc.direct_conv_rect(img, d, None, 0, 1)
+    assert np.array_equal(y[0, 0, :, :5], img[0, 0, :, 1:].astype(np.float64)) and not y[0, 0, :, 5].any()
