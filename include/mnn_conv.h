@@ -153,7 +153,7 @@ typedef struct {
     int paper_n_hat;
     unsigned long long paper_mul[4];
     int strassen;                    /* 1 when the plan runs one Strassen level (alpha = 1, seven products) */
-    int reserved0;
+    int rect;                        /* plans of mnn_conv_plan_rect: 1 = kernel 1 x k, 2 = kernel k x 1; else 0 */
 } mnn_conv_info;
 
 /* Plan one layer with groups = 1, relu = 1, accuracy class TF32, everything else
@@ -165,6 +165,17 @@ MNN_API mnn_conv_plan_t mnn_conv_plan(int N, int Cin, int Cout, int H, int W, in
 /* Same with explicit options (opts may be NULL = all defaults incl. relu = 0). */
 MNN_API mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k,
                                  int stride, int pad, int dilation, const mnn_conv_opts* opts);
+
+/* Rectangular kernels 1 x k and k x 1 (the paper's Section 4.2 names the 1 x 7 and 7 x 1 layers of Inception-v3
+ * as a case other engines handle badly): w is [Cout][Cin][kh][kw] with kh = 1 or kw = 1 and the other one k in
+ * {2, 3, 5, 7}; stride 1, no dilation, one group, padding given per axis; OH = H + 2 pad_h - kh + 1, OW likewise.
+ * The layer runs as a ONE-dimensional Winograd F(m, k) along the kernel's long axis (Eq. 6 with the identity on
+ * the other axis: alpha = m + k - 1 transform positions) through the same tensor-core contraction.  opts as for
+ * mnn_conv_plan_ex (relu, precision, operand, passes, force_m, points_id are read; force_m = 0 takes m = 4,
+ * or 2 where m + k - 1 would pass 10; operand AUTO takes BF16 hi + lo under the TF32 accuracy class).
+ * The plan is used with the same mnn_conv_* calls as any other; info.alpha is the number of transform positions. */
+MNN_API mnn_conv_plan_t mnn_conv_plan_rect(int N, int Cin, int Cout, int H, int W, int kh, int kw, int pad_h, int pad_w,
+                                           const mnn_conv_opts* opts);
 
 /* Copy the plan's decisions into *info (host). */
 MNN_API int mnn_conv_plan_query(mnn_conv_plan_t plan, mnn_conv_info* info);

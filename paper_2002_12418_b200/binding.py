@@ -25,7 +25,7 @@ COST_INADMISSIBLE = 0xFFFFFFFFFFFFFFFF
 ALGO_NAMES = {ALGO_WINOGRAD: "winograd", ALGO_GEMM: "gemm", ALGO_DIRECT: "direct"}
 OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "fp32ref", 0: "-"}
 
-EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_query", "mnn_conv_set_workspace",
+EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_rect", "mnn_conv_plan_query", "mnn_conv_set_workspace",
             "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
             "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_strassen_rule", "mnn_calibrate",
             "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error",
@@ -55,7 +55,7 @@ class ConvInfo(ctypes.Structure):
                 ("chosen_candidate", ctypes.c_int), ("gemm_lhs", ctypes.c_int),
                 ("cost_ps", ctypes.c_ulonglong * N_CANDIDATES),
                 ("fused", ctypes.c_int), ("paper_n_hat", ctypes.c_int), ("paper_mul", ctypes.c_ulonglong * 4),
-                ("strassen", ctypes.c_int), ("reserved0", ctypes.c_int)]
+                ("strassen", ctypes.c_int), ("rect", ctypes.c_int)]
 
 
 class LayerDesc(ctypes.Structure):
@@ -96,6 +96,8 @@ def lib():
         L.mnn_conv_plan.restype = p
         L.mnn_conv_plan_ex.argtypes = [i] * 9 + [ctypes.POINTER(ConvOpts)]
         L.mnn_conv_plan_ex.restype = p
+        L.mnn_conv_plan_rect.argtypes = [i] * 9 + [ctypes.POINTER(ConvOpts)]
+        L.mnn_conv_plan_rect.restype = p
         L.mnn_conv_plan_query.argtypes = [p, ctypes.POINTER(ConvInfo)]
         L.mnn_conv_plan_query.restype = i
         L.mnn_conv_set_workspace.argtypes = [p, p, ll]
@@ -178,6 +180,13 @@ def mnn_conv_plan(N, Cin, Cout, H, W, k, stride, pad, dilation):
 def mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation, opts: ConvOpts | None):
     h = lib().mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation,
                                ctypes.byref(opts) if opts is not None else None)
+    if not h:
+        raise MnnError(MNN_EINVAL, mnn_last_error())
+    return h
+
+
+def mnn_conv_plan_rect(N, Cin, Cout, H, W, kh, kw, pad_h, pad_w, opts: ConvOpts | None):
+    h = lib().mnn_conv_plan_rect(N, Cin, Cout, H, W, kh, kw, pad_h, pad_w, ctypes.byref(opts) if opts is not None else None)
     if not h:
         raise MnnError(MNN_EINVAL, mnn_last_error())
     return h
@@ -371,13 +380,16 @@ class ConvLayerRunner:
     stream through mnn_conv_run; nothing here computes."""
 
     def __init__(self, N, Cin, Cout, H, W, k, stride=1, pad=0, dilation=1, opts: ConvOpts | None = None,
-                 device="cuda:0"):
+                 device="cuda:0", plan=None):
         import torch
         self.torch = torch
         self.device = torch.device(device)
         self.shape = (N, Cin, Cout, H, W, k, stride, pad, dilation)
-        self.plan = mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation, opts) if opts is not None \
-            else mnn_conv_plan(N, Cin, Cout, H, W, k, stride, pad, dilation)
+        if plan is not None:
+            self.plan = plan               # e.g. from mnn_conv_plan_rect; owned by the runner from here on
+        else:
+            self.plan = mnn_conv_plan_ex(N, Cin, Cout, H, W, k, stride, pad, dilation, opts) if opts is not None \
+                else mnn_conv_plan(N, Cin, Cout, H, W, k, stride, pad, dilation)
         self.info = mnn_conv_plan_query(self.plan)
         self.workspace = None
         if self.info.workspace_bytes > 0:

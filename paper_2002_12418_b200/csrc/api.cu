@@ -14,6 +14,7 @@
 #include "planner.h"
 #include "strassen.h"
 #include "wino_fused.h"
+#include "wino_rect.h"
 
 using namespace mnnb;
 
@@ -58,6 +59,8 @@ struct mnn_conv_plan_s {
     const float* prepared_w = nullptr;
     UmmaContract uc;
     bool strassen = false;           // GEMM scheme through one Strassen level: seven half-size products
+    int rect = 0;                    // 1: kernel 1 x k, 2: kernel k x 1 (one-dimensional Winograd along the long axis)
+    int pad_h = 0, pad_w = 0;        // rectangular plans: padding per axis (s.pad is unused there)
     bool fused = false;              // Winograd F(2x2,3x3) as the single fused kernel: the workspace holds U only
     FusedWino fw;
     // optional per-launch timing
@@ -98,7 +101,16 @@ void layout_workspace(mnn_conv_plan_t p)
         return;
     }
     long long off = kStatusBytes;
-    if (d.algo == MNN_ALGO_WINOGRAD) {
+    if (p->rect) {
+        const long long n_seg = p->rect == 1 ? (s.OW + d.m - 1) / d.m : (s.OH + d.m - 1) / d.m;
+        p->cin_pad = (int)align_up(s.Cin, 8);
+        p->chunk_tiles = p->rect == 1 ? (long long)s.N * s.OH * n_seg : (long long)s.N * n_seg * s.OW;
+        p->m_row_stride = (int)align_up(p->chunk_tiles, 32);
+        p->u_bytes = align_up((long long)d.alpha * s.Cout * p->cin_pad * eb, 2048);
+        p->v_bytes = align_up((long long)d.alpha * p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->m_bytes = align_up((long long)d.alpha * s.Cout * p->m_row_stride * 4, 1024);
+        p->launches_per_run = 3;
+    } else if (d.algo == MNN_ALGO_WINOGRAD) {
         const long long a2 = (long long)d.alpha * d.alpha;
         const long long th = (s.OH + d.m - 1) / d.m, tw = (s.OW + d.m - 1) / d.m;
         p->cin_pad = (int)align_up(s.Cin, 8);
@@ -273,6 +285,102 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
     return p;
 }
 
+mnn_conv_plan_t mnn_conv_plan_rect(int N, int Cin, int Cout, int H, int W, int kh, int kw, int pad_h, int pad_w,
+                                   const mnn_conv_opts* opts)
+{
+    mnn_conv_opts o;
+    std::memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    if (N <= 0 || Cin <= 0 || Cout <= 0 || H <= 0 || W <= 0 || kh <= 0 || kw <= 0 || pad_h < 0 || pad_w < 0) {
+        fail(MNN_EINVAL, "sizes must be positive and paddings non-negative");
+        return nullptr;
+    }
+    const int k = kh > kw ? kh : kw;
+    if ((kh != 1 && kw != 1) || k == 1 || !(k == 2 || k == 3 || k == 5 || k == 7) || (o.groups != 0 && o.groups != 1)) {
+        fail(MNN_EUNSUPPORTED, "rectangular plans take 1 x k or k x 1 kernels with k in {2,3,5,7} and one group; "
+                               "square kernels go through mnn_conv_plan_ex");
+        return nullptr;
+    }
+    if (o.precision != MNN_PREC_TF32 && o.precision != MNN_PREC_BF16) {
+        fail(MNN_EINVAL, "precision must be MNN_PREC_TF32 or MNN_PREC_BF16");
+        return nullptr;
+    }
+    const int OH = H + 2 * pad_h - kh + 1, OW = W + 2 * pad_w - kw + 1;
+    if (OH <= 0 || OW <= 0) {
+        fail(MNN_EINVAL, "the kernel does not fit the padded input");
+        return nullptr;
+    }
+    int m = o.force_m ? o.force_m : (4 + k - 1 <= kRectMaxAlpha ? 4 : 2);
+    if (!(m == 2 || m == 4 || m == 6) || m + k - 1 > kRectMaxAlpha) {
+        fail(MNN_EUNSUPPORTED, "rectangular plans take m in {2,4,6} with m + k - 1 <= 10");
+        return nullptr;
+    }
+    if (o.operand == MNN_OPERAND_FP32_REF || o.operand < 0 || o.operand > MNN_OPERAND_FP32_REF ||
+        !(o.passes == 0 || o.passes == 1 || o.passes == 3) || o.points_id < 0 || o.points_id > MNN_POINTS_MIXED) {
+        fail(MNN_EINVAL, "an option is outside its range");
+        return nullptr;
+    }
+    // The accuracy model is the two-dimensional one (an upper bound for one dimension): single-pass operands where
+    // it admits them for the class, else the hi + lo split.
+    const long long gate = (o.precision == MNN_PREC_BF16 ? 10000 : 1000) * kGateNumerator / kGateDenominator;
+    int operand = o.operand, passes = o.passes;
+    if (operand == MNN_OPERAND_AUTO) {
+        operand = MNN_OPERAND_BF16;
+        if (passes == 0) {
+            long long ppm1 = 0;
+            best_points(m, k, operand, 1, &ppm1);
+            passes = (ppm1 >= 0 && ppm1 <= gate) ? 1 : 3;
+        }
+    } else if (passes == 0) {
+        passes = 1;
+    }
+    long long ppm = 0;
+    const int pid = o.points_id ? o.points_id : best_points(m, k, operand, passes, &ppm);
+    if (o.points_id) ppm = accuracy_ppm(m, k, pid, operand, passes);
+    WinogradMatrices wm;
+    if (pid == 0 || !generate_winograd(m, k, pid, &wm)) {
+        fail(MNN_EUNSUPPORTED, "no transform matrices for this (m, k, points)");
+        return nullptr;
+    }
+    mnn_conv_plan_t p = new (std::nothrow) mnn_conv_plan_s();
+    if (!p) {
+        fail(MNN_EINVAL, "out of host memory");
+        return nullptr;
+    }
+    LayerShape s;
+    s.N = N; s.Cin = Cin; s.Cout = Cout; s.H = H; s.W = W; s.k = k; s.stride = 1; s.pad = 0; s.dil = 1;
+    s.groups = 1; s.relu = o.relu ? 1 : 0; s.OH = OH; s.OW = OW;
+    o.groups = 1;
+    p->s = s;
+    p->o = o;
+    p->rect = kh == 1 ? 1 : 2;
+    p->pad_h = pad_h;
+    p->pad_w = pad_w;
+    for (int i = 0; i < MNN_N_CANDIDATES; ++i) p->d.cost_ps[i] = MNN_COST_INADMISSIBLE;
+    p->d.algo = MNN_ALGO_WINOGRAD;
+    p->d.m = m;
+    p->d.alpha = m + k - 1;
+    p->d.operand = operand;
+    p->d.passes = passes;
+    p->d.points_id = pid;
+    p->d.chunk_images = N;
+    p->d.n_chunks = 1;
+    p->d.chosen = -1;
+    p->d.error_ppm = ppm;
+    std::memset(&p->mats, 0, sizeof(p->mats));
+    std::memcpy(p->mats.At, wm.At32.data(), wm.At32.size() * sizeof(float));
+    std::memcpy(p->mats.G, wm.G32.data(), wm.G32.size() * sizeof(float));
+    std::memcpy(p->mats.Bt, wm.Bt32.data(), wm.Bt32.size() * sizeof(float));
+    layout_workspace(p);
+    if (p->v_bytes + p->m_bytes > (4ll << 30) || (long long)N * Cin * H * W >= (1ll << 40) ||
+        (long long)N * Cout * OH * OW >= (1ll << 40)) {
+        fail(MNN_EUNSUPPORTED, "layer too large for one pass of the rectangular path: split the batch");
+        delete p;
+        return nullptr;
+    }
+    return p;
+}
+
 mnn_conv_plan_t mnn_conv_plan(int N, int Cin, int Cout, int H, int W, int k, int stride, int pad, int dilation)
 {
     mnn_conv_opts o;
@@ -317,6 +425,7 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     for (int i = 0; i < MNN_N_CANDIDATES; ++i) info->cost_ps[i] = p->d.cost_ps[i];
     info->fused = p->fused ? 1 : 0;
     info->strassen = p->strassen ? 1 : 0;
+    info->rect = p->rect;
     if (p->strassen) info->predicted_error_ppm = 3 * p->d.error_ppm;
     info->paper_n_hat = p->d.paper_n_hat;
     for (int i = 0; i < 4; ++i) info->paper_mul[i] = p->d.paper_mul[i];
@@ -328,6 +437,9 @@ static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
 {
     const int alpha2 = p->d.algo == MNN_ALGO_WINOGRAD ? p->d.alpha * p->d.alpha : 1;
     if (p->fused) return fused_wino_setup(&p->fw, p->s.Cout, p->s.Cin, u_hi(p), why);
+    if (p->rect)
+        return umma_contract_setup(&p->uc, p->store_mode, p->d.alpha, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p),
+                                   v_hi(p), v_lo(p), why);
     if (p->strassen)
         return umma_contract_setup(&p->uc, p->store_mode, 7, p->s.Cout / 2, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
                                    v_lo(p), why);
@@ -430,11 +542,26 @@ static StrassenGeom strassen_geom(mnn_conv_plan_t p)
     return g;
 }
 
+static RectGeom rect_geom(mnn_conv_plan_t p)
+{
+    RectGeom g;
+    g.N = p->s.N; g.Cin = p->s.Cin; g.Cout = p->s.Cout; g.H = p->s.H; g.W = p->s.W; g.OH = p->s.OH; g.OW = p->s.OW;
+    g.k = p->s.k; g.along_w = p->rect == 1 ? 1 : 0; g.pad_h = p->pad_h; g.pad_w = p->pad_w;
+    g.m = p->d.m; g.alpha = p->d.alpha;
+    g.n_seg = p->rect == 1 ? (p->s.OW + g.m - 1) / g.m : (p->s.OH + g.m - 1) / g.m;
+    g.cin_pad = p->cin_pad;
+    g.tiles = p->chunk_tiles;
+    g.m_row_stride = p->m_row_stride;
+    return g;
+}
+
 static int do_weights(mnn_conv_plan_t p, const float* w, cudaStream_t st)
 {
     cudaError_t e;
     LaunchTimer lt(p, st, 0);
-    if (p->strassen)
+    if (p->rect)
+        e = launch_rect_weights(w, u_hi(p), u_lo(p), rect_geom(p), p->store_mode, p->mats, st);
+    else if (p->strassen)
         e = launch_strassen_weights(w, u_hi(p), u_lo(p), strassen_geom(p), p->store_mode, st);
     else if (p->fused)
         e = launch_fused_wino_weights(w, u_hi(p), p->s.Cout, p->s.Cin, p->mats, st);
@@ -488,6 +615,27 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
     }
     const bool reference = d.operand == MNN_OPERAND_FP32_REF;
 
+    if (p->rect) {
+        const RectGeom g = rect_geom(p);
+        if (reference) return fail(MNN_EUNSUPPORTED, "rectangular kernels run on the tensor-core contraction only");
+        if (mask & MNN_STAGE_INPUT) {
+            LaunchTimer lt(p, st, 1);
+            e = launch_rect_input(x, v_hi(p), v_lo(p), g, p->store_mode, p->mats, st);
+            if (e != cudaSuccess) return fail_cuda(e, "one-dimensional input transform");
+        }
+        if (mask & MNN_STAGE_CONTRACT) {
+            ContractEpilogue epi = {0, m_buf(p), p->m_row_stride, nullptr, nullptr, 0, 1};
+            LaunchTimer lt(p, st, 2);
+            e = launch_contract_umma(p->uc, g.tiles, epi, status_word(p), st);
+            if (e != cudaSuccess) return fail_cuda(e, "Winograd contraction");
+        }
+        if (mask & MNN_STAGE_OUTPUT) {
+            LaunchTimer lt(p, st, 3);
+            e = launch_rect_output(m_buf(p), bias, y, g, s.relu, p->mats, st);
+            if (e != cudaSuccess) return fail_cuda(e, "one-dimensional output transform");
+        }
+        return MNN_OK;
+    }
     if (p->strassen) {
         const StrassenGeom g = strassen_geom(p);
         if (reference) return fail(MNN_EUNSUPPORTED, "Strassen runs on the tensor-core contraction only");
