@@ -10,6 +10,7 @@
 
 #include "../../include/mnn_conv.h"
 #include "generator.h"
+#include "contract_umma.h"
 #include "kernels.h"
 #include "planner.h"
 #include "strassen.h"

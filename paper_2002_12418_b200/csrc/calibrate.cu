@@ -11,6 +11,7 @@
 
 #include "../../include/mnn_conv.h"
 #include "generator.h"
+#include "contract_umma.h"
 #include "kernels.h"
 #include "planner.h"
 #include "wino_fused.h"

@@ -30,6 +30,7 @@
 // to nearest).
 #include <cuda_bf16.h>
 
+#include "contract_umma.h"
 #include "kernels.h"
 #include "planner.h"
 #include "umma.cuh"
@@ -61,7 +62,24 @@ struct KernelParams {
 // status codes written on a bounded wait that ran out
 constexpr int kErrProducerWait = 1, kErrMmaWaitFull = 2, kErrMmaWaitTmem = 3, kErrEpilogueWait = 4;
 
-template <int KIND>
+// Shared-memory descriptor of a K-major operand tile whose rows are SW bytes long and SW-byte swizzled.
+template <int SW>
+__device__ __forceinline__ uint64_t desc_k(uint32_t smem_addr)
+{
+    if (SW == 128) return ptx::smem_desc_k128(smem_addr);
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(512 >> 4) << 32;                         // 8-row groups of 64-byte rows
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;                                  // 64-byte swizzle
+    return d;
+}
+
+// SW = bytes of K per shared-memory row of an operand tile (the swizzle span): 128, or 64 where 128-byte rows
+// would leave room for two pipeline stages only (hi + lo operands with wide channel blocks): the same bytes
+// in flight in twice as many stages keep the tensor core fed across the TMA latency.
+template <int KIND, int SW>
 __global__ void __launch_bounds__(kThreads, 1)
 contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_constant__ CUtensorMap map_v_lo,
                      const __grid_constant__ CUtensorMap map_u_hi, const __grid_constant__ CUtensorMap map_u_lo,
@@ -80,8 +98,8 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = kTileM * kSwizzleBytes;                 // one V tile (128 tiles)
-    const uint32_t b_bytes = (uint32_t)p.bn * kSwizzleBytes;         // one U tile (bn output channels)
+    const uint32_t a_bytes = kTileM * SW;                            // one V tile (128 tiles)
+    const uint32_t b_bytes = (uint32_t)p.bn * SW;                    // one U tile (bn output channels)
     const uint32_t split = p.passes == 3 ? 2u : 1u;
     const uint32_t stage_bytes = (a_bytes + b_bytes) * split;
     // stage layout: [A_hi][A_lo?][B_hi][B_lo?]
@@ -118,7 +136,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");          // the epilogue warps only
     }
 
-    const int k_elems = KIND == 0 ? 32 : 64;         // elements of K per 128-byte row
+    const int k_elems = (KIND == 0 ? 32 : 64) * SW / 128;   // elements of K per shared-memory row
 
     if (warp == 0) {
         if (lane == 0) {
@@ -190,15 +208,15 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     ptx::tc_fence_after();
                     const uint32_t sbase = smem_base + stage * stage_bytes;
 #pragma unroll
-                    for (int ks = 0; ks < kSwizzleBytes / 32; ++ks) {
+                    for (int ks = 0; ks < SW / 32; ++ks) {
                         // K-major: 8 K elements are 32 bytes along the row; MN-major: 8 rows of 128 bytes
-                        const uint64_t a_hi = p.a_mn ? ptx::smem_desc_mn128_b32(sbase + ks * 1024, 4096)
-                                                     : ptx::smem_desc_k128(sbase + ks * 32);
-                        const uint64_t b_hi = ptx::smem_desc_k128(sbase + off_b_hi + ks * 32);
+                        const uint64_t a_hi = (SW == 128 && p.a_mn) ? ptx::smem_desc_mn128_b32(sbase + ks * 1024, 4096)
+                                                                    : desc_k<SW>(sbase + ks * 32);
+                        const uint64_t b_hi = desc_k<SW>(sbase + off_b_hi + ks * 32);
                         ptx::mma_ss<KIND>(d_tmem, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
                         if (split == 2) {
-                            const uint64_t a_lo = ptx::smem_desc_k128(sbase + off_a_lo + ks * 32);
-                            const uint64_t b_lo = ptx::smem_desc_k128(sbase + off_b_lo + ks * 32);
+                            const uint64_t a_lo = desc_k<SW>(sbase + off_a_lo + ks * 32);
+                            const uint64_t b_lo = desc_k<SW>(sbase + off_b_lo + ks * 32);
                             ptx::mma_ss<KIND>(d_tmem, a_lo, b_hi, idesc, 1u);
                             ptx::mma_ss<KIND>(d_tmem, a_hi, b_lo, idesc, 1u);
                         }
@@ -372,17 +390,28 @@ EncodeTiledFn get_encode_fn()
 }  // namespace
 
 // 3-D map over [planes][rows][k] (k contiguous), box = [1][box_rows][128 bytes of k], 128-byte swizzle.
+static bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
+                                  long long plane_stride_elems, int box_rows, int sw);
+
 bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
                         long long plane_stride_elems, int box_rows)
+{
+    return encode_operand_map_sw(map, base, elem_bytes, k_len, rows, planes, plane_stride_elems, box_rows, kSwizzleBytes);
+}
+
+// The same with rows of `sw` bytes (128 or 64) and the matching swizzle.
+static bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
+                                  long long plane_stride_elems, int box_rows, int sw)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)k_len, (cuuint64_t)rows, (cuuint64_t)planes};
     const cuuint64_t strides[2] = {(cuuint64_t)k_len * elem_bytes, (cuuint64_t)plane_stride_elems * elem_bytes};
-    const cuuint32_t box[3] = {(cuuint32_t)(kSwizzleBytes / elem_bytes), (cuuint32_t)box_rows, 1};
+    const cuuint32_t box[3] = {(cuuint32_t)(sw / elem_bytes), (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-    CUresult r = fn(map, dt, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    CUresult r = fn(map, dt, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    sw == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -451,10 +480,15 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     if (e != cudaSuccess) return e;
     // output channels per work item (MMA N) and the channel blocks
     contract_tiling((tiles_capacity + kTileM - 1) / kTileM, alpha2, Cout, uc->num_sms, &uc->bn, &uc->n_co_blocks);
-    const int k_elems = kSwizzleBytes / eb;
-    uc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
     const int split = uc->passes == 3 ? 2 : 1;
-    const int stage_bytes = (kTileM * kSwizzleBytes + uc->bn * kSwizzleBytes) * split;
+    // rows of 128 bytes unless that leaves fewer than three stages and the K loop is long (at least four
+    // 128-byte blocks; measured: 512 channels BF16 hi + lo 0.604 -> 0.576 ms, shorter loops lose)
+    int sw = kSwizzleBytes;
+    if (!uc->a_mn && (kSmemBudget - 1024) / ((kTileM + uc->bn) * sw * split) < 3 && cin_pad * eb >= 4 * sw) sw = 64;
+    uc->stages_sw = sw;
+    const int k_elems = sw / eb;
+    uc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
+    const int stage_bytes = (kTileM * sw + uc->bn * sw) * split;
     int stages = (kSmemBudget - 1024) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) {
@@ -470,11 +504,11 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     uc->tmem_cols = cols;
 
     const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
-    bool ok = (uc->a_mn || encode_operand_map(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM)) &&
-              encode_operand_map(&uc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
+    bool ok = (uc->a_mn || encode_operand_map_sw(&uc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM, sw)) &&
+              encode_operand_map_sw(&uc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, uc->bn, sw);
     if (ok && split == 2)
-        ok = encode_operand_map(&uc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM) &&
-             encode_operand_map(&uc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, uc->bn);
+        ok = encode_operand_map_sw(&uc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM, sw) &&
+             encode_operand_map_sw(&uc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, uc->bn, sw);
     if (!ok) {
         *why = "cuTensorMapEncodeTiled failed or is unavailable";
         return cudaErrorInvalidValue;
@@ -484,12 +518,11 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
         uc->map_v_lo = uc->map_v_hi;
         uc->map_u_lo = uc->map_u_hi;
     }
-    auto k0 = contract_umma_kernel<0>;
-    auto k1 = contract_umma_kernel<1>;
-    e = cudaFuncSetAttribute(k0, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-    if (e != cudaSuccess) return e;
+    for (auto kern : {contract_umma_kernel<0, 128>, contract_umma_kernel<1, 128>, contract_umma_kernel<0, 64>,
+                      contract_umma_kernel<1, 64>}) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (e != cudaSuccess) return e;
+    }
     uc->ready = true;
     return cudaSuccess;
 }
@@ -567,7 +600,7 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.epi = epi;
     p.status = status;
     const long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    return launch_overlapped(contract_umma_kernel<0>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
+    return launch_overlapped(contract_umma_kernel<0, 128>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
                              map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
 }
 
@@ -597,11 +630,10 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     p.epi = epi;
     p.status = status;
     long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    if (uc.kind == 0)
-        return launch_overlapped(contract_umma_kernel<0>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
-                                 uc.map_v_hi, uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
-    return launch_overlapped(contract_umma_kernel<1>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
-                             uc.map_v_hi, uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
+    auto kern = uc.kind == 0 ? (uc.stages_sw == 64 ? contract_umma_kernel<0, 64> : contract_umma_kernel<0, 128>)
+                             : (uc.stages_sw == 64 ? contract_umma_kernel<1, 64> : contract_umma_kernel<1, 128>);
+    return launch_overlapped(kern, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream, uc.map_v_hi,
+                             uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
 }
 
 }  // namespace mnnb
