@@ -52,7 +52,7 @@ enum { MNN_ALGO_AUTO = 0, MNN_ALGO_WINOGRAD = 1, MNN_ALGO_GEMM = 2, MNN_ALGO_DIR
 enum { MNN_PREC_TF32 = 0, MNN_PREC_BF16 = 1 };             /* accuracy class */
 enum { MNN_OPERAND_AUTO = 0, MNN_OPERAND_TF32 = 1, MNN_OPERAND_BF16 = 2, MNN_OPERAND_FP32_REF = 3 };
 enum { MNN_POINTS_AUTO = 0, MNN_POINTS_PAPER = 1, MNN_POINTS_UNIT = 2, MNN_POINTS_MIXED = 3 };
-enum { MNN_GEMM_LHS_AUTO = 0, MNN_GEMM_LHS_PATCHES = 1, MNN_GEMM_LHS_X = 2 };
+enum { MNN_GEMM_LHS_AUTO = 0, MNN_GEMM_LHS_PATCHES = 1, MNN_GEMM_LHS_X = 2, MNN_GEMM_LHS_IMPLICIT = 3 };
 enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_STAGE_OUTPUT = 8,
        MNN_STAGE_ALL = 15 };
 
@@ -88,8 +88,11 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
  *              only for 1x1 stride-1 unpadded ungrouped layers with H*W >= 32 and a
  *              multiple of 4 and single-pass TF32 operands, where the tensor core drops
  *              the low 13 mantissa bits of x (truncation) instead of a rounded copy being
- *              stored.  AUTO = the planner takes the cheaper where X applies.  Asking
- *              for X where it does not apply fails the plan.
+ *              stored.  IMPLICIT: no patch matrix either, for any k / stride / padding /
+ *              dilation: producer warps of the GEMM kernel gather the patches into the
+ *              shared-memory operand tile themselves (single-pass TF32 operands, rounded
+ *              to nearest).  AUTO = the planner takes the cheapest that applies.  Asking
+ *              for X or IMPLICIT where it does not apply fails the plan.
  *   fused      Winograd F(2x2, 3x3) as ONE kernel (input transform, contraction and output
  *              transform fused; the transformed tensors V and M never reach device memory):
  *              0 = the planner weighs it against the other candidates, 1 = never,
@@ -147,7 +150,7 @@ typedef struct {
     long long u_offset, u_bytes, v_offset, v_bytes, m_offset, m_bytes;
     long long predicted_error_ppm;   /* accuracy model's relative L2 error x 1e6 for the choice */
     int chosen_candidate;            /* index into cost_ps, -1 when the choice was forced outside the list */
-    int gemm_lhs;                    /* GEMM scheme: MNN_GEMM_LHS_PATCHES or MNN_GEMM_LHS_X as planned, else 0 */
+    int gemm_lhs;                    /* GEMM scheme: MNN_GEMM_LHS_PATCHES, _X or _IMPLICIT as planned, else 0 */
     unsigned long long cost_ps[MNN_N_CANDIDATES];
     int fused;                       /* 1 when the plan is the single fused Winograd kernel (no V, no M) */
     int paper_n_hat;
@@ -289,7 +292,9 @@ MNN_API int mnn_strassen_rule(long long m, long long n, long long k);
  * consts[11] picoseconds the fused kernel's tensor work takes per block of 32 input channels of one work item
  * consts[12] picoseconds of epilogue per work item of the fused kernel
  *            (consts[10] or [11] = 0: the fused kernel is never chosen by the planner)
- * consts[13..15] reserved (0).
+ * consts[13] attoseconds per patch element gathered by the implicit GEMM's producer warps, per SM
+ *            (0 = the planner never takes the implicit left operand by itself)
+ * consts[14..15] reserved (0).
  * mnn_calibrate measures them on the current device (launches micro-benchmarks and
  * synchronises; allocates and frees its own scratch) and installs them;
  * mnn_set_calibration installs a frozen record so that plans are reproducible;

@@ -37,7 +37,7 @@ from dataclasses import dataclass, field
 ALGO_WINOGRAD, ALGO_GEMM, ALGO_DIRECT = 1, 2, 3
 OPERAND_TF32, OPERAND_BF16, OPERAND_FP32_REF = 1, 2, 3
 PREC_TF32, PREC_BF16 = 0, 1
-LHS_PATCHES, LHS_X = 1, 2
+LHS_PATCHES, LHS_X, LHS_IMPLICIT = 1, 2, 3
 INADMISSIBLE = 2 ** 64 - 1
 SATURATED = 2 ** 64 - 2
 MAX_CHUNK_BYTES = 4 << 30          # V + M of one chunk may not exceed this, whatever the cost says
@@ -161,7 +161,11 @@ def gemm_may_read_x(L: Layer, operand: int, passes: int) -> bool:
             and passes == 1 and L.H * L.W >= 32 and (L.H * L.W) % 4 == 0)
 
 
-def gemm_cost(L: Layer, operand: int, lhs_x: bool, c) -> int:
+def gemm_cost(L: Layer, operand: int, lhs, c) -> int:
+    """lhs: LHS_PATCHES (gather kernel + GEMM), LHS_X / True (the GEMM reads x itself), LHS_IMPLICIT (the patches are
+    gathered by producer warps inside the GEMM kernel)."""
+    lhs_x = lhs is True or lhs == LHS_X
+    implicit = lhs is not True and lhs == LHS_IMPLICIT
     b = _bytes_of(operand)
     Kp = cdiv(L.Cin * L.k * L.k, 8) * 8
     T = L.N * L.OH * L.OW
@@ -181,6 +185,12 @@ def gemm_cost(L: Layer, operand: int, lhs_x: bool, c) -> int:
     deliver_ps = (128 * 128 + bn * 128) * 16
     mma_ps = sat(2 * 128 * bn * k_elems * _tensor_rate(c, operand) * sms // 1_000_000)
     drain_ps = 128 * bn * 4 * 45
+    if implicit:
+        # only the weight tile is delivered; the gather of 128 x 32 patch elements (c[13] attoseconds each) paces a block too
+        # (c[13] is measured on the tap-major gather, Cin a multiple of 32; other channel counts gather element-wise, about 2x)
+        block_ps = max(bn * 128 * 16, mma_ps, sat(128 * 32 * c[13] * (1 if L.Cin % 32 == 0 else 2) // 1_000_000))
+        item_i = max(k_blocks * block_ps, drain_ps + 500_000)
+        return kernel_ps(c, mem_as=(x_bytes + u_bytes + y_bytes) * c[0], tensor_as=(rounds * item_i + drain_ps) * 1_000_000)
     item_ps = max(k_blocks * max(deliver_ps, mma_ps), drain_ps + 500_000)
     serial_as = (rounds * item_ps + drain_ps) * 1_000_000
     if lhs_x:
@@ -315,15 +325,29 @@ def plan(L: Layer, o: Options, c, ppm) -> Choice:
             if p > gate and not (o.operand != 0 and o.force_algo == ALGO_GEMM):
                 continue
             x_ok = gemm_may_read_x(L, operand, passes)
+            implicit_ok = operand == OPERAND_TF32 and passes == 1
             if o.gemm_lhs == LHS_X and not x_ok:
                 continue
-            cost_p = gemm_cost(L, operand, False, c)
-            cost_x = gemm_cost(L, operand, True, c) if x_ok else INADMISSIBLE
-            take_x = o.gemm_lhs == LHS_X or (o.gemm_lhs == 0 and x_ok and cost_x < cost_p)
-            if take_x:
+            if o.gemm_lhs == LHS_IMPLICIT and not implicit_ok:
+                continue
+            costs = {LHS_PATCHES: gemm_cost(L, operand, LHS_PATCHES, c)}
+            if x_ok:
+                costs[LHS_X] = gemm_cost(L, operand, LHS_X, c)
+            if implicit_ok:
+                costs[LHS_IMPLICIT] = gemm_cost(L, operand, LHS_IMPLICIT, c)
+            # left operand: as asked for, else the cheapest that applies (patch matrix, x itself, implicit gather;
+            # earlier in this order on ties; the implicit gather only once its rate constant is known)
+            lhs = o.gemm_lhs
+            if lhs == 0:
+                lhs = LHS_PATCHES
+                if x_ok and costs[LHS_X] < costs[lhs]:
+                    lhs = LHS_X
+                if implicit_ok and c[13] > 0 and costs[LHS_IMPLICIT] < costs[lhs]:
+                    lhs = LHS_IMPLICIT
+            if lhs == LHS_X:
                 p = max(p, LHS_X_ERROR_PPM)
-            side[i] = dict(lhs=LHS_X if take_x else LHS_PATCHES, ppm=p)
-            ch.cost_ps[i] = cost_x if take_x else cost_p
+            side[i] = dict(lhs=lhs, ppm=p)
+            ch.cost_ps[i] = costs[lhs]
             continue
         # Winograd
         fused = i == FUSED_SLOT

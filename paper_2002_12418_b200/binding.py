@@ -17,7 +17,7 @@ ALGO_AUTO, ALGO_WINOGRAD, ALGO_GEMM, ALGO_DIRECT = 0, 1, 2, 3
 PREC_TF32, PREC_BF16 = 0, 1
 OPERAND_AUTO, OPERAND_TF32, OPERAND_BF16, OPERAND_FP32_REF = 0, 1, 2, 3
 POINTS_AUTO, POINTS_PAPER, POINTS_UNIT, POINTS_MIXED = 0, 1, 2, 3
-GEMM_LHS_AUTO, GEMM_LHS_PATCHES, GEMM_LHS_X = 0, 1, 2
+GEMM_LHS_AUTO, GEMM_LHS_PATCHES, GEMM_LHS_X, GEMM_LHS_IMPLICIT = 0, 1, 2, 3
 FUSED_AUTO, FUSED_NEVER, FUSED_ONLY = 0, 1, 2
 STAGE_WEIGHT, STAGE_INPUT, STAGE_CONTRACT, STAGE_OUTPUT, STAGE_ALL = 1, 2, 4, 8, 15
 N_CANDIDATES, N_CONSTS = 16, 16

@@ -10,6 +10,7 @@
 
 #include "../../include/mnn_conv.h"
 #include "generator.h"
+#include "implicit_gemm.h"
 #include "contract_umma.h"
 #include "kernels.h"
 #include "planner.h"
@@ -52,6 +53,8 @@ struct mnn_conv_plan_s {
     long long u_offset = 0, u_bytes = 0, v_offset = 0, v_bytes = 0, m_offset = 0, m_bytes = 0, workspace_bytes = 0;
     int launches_per_run = 1;
     bool gemm_x = false;             // GEMM scheme with x itself as the left operand: no V, one launch
+    bool gemm_implicit = false;      // GEMM scheme with the patches gathered inside the GEMM kernel: no V, one launch
+    ImplicitGemm ig;
     TransformMatrices mats;
     // run-time state
     char* ws = nullptr;              // status word and U (persistent part), and V, M unless tws is set
@@ -137,9 +140,11 @@ void layout_workspace(mnn_conv_plan_t p)
         p->m_row_stride = 0;
         p->u_bytes = align_up((long long)s.Cout * p->cin_pad * eb, 2048);
         p->gemm_x = d.gemm_lhs == MNN_GEMM_LHS_X;
-        p->v_bytes = p->gemm_x ? 0 : align_up(p->chunk_tiles * p->cin_pad * eb, 2048);
+        p->gemm_implicit = d.gemm_lhs == MNN_GEMM_LHS_IMPLICIT;
+        const bool no_v = p->gemm_x || p->gemm_implicit;
+        p->v_bytes = no_v ? 0 : align_up(p->chunk_tiles * p->cin_pad * eb, 2048);
         p->m_bytes = 0;
-        p->launches_per_run = p->gemm_x ? 1 : 2;
+        p->launches_per_run = no_v ? 1 : 2;
     }
     p->u_offset = off;
     off += p->u_bytes;
@@ -210,7 +215,7 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
     }
     if (o.operand < 0 || o.operand > MNN_OPERAND_FP32_REF || !(o.passes == 0 || o.passes == 1 || o.passes == 3) ||
         o.force_algo < 0 || o.force_algo > MNN_ALGO_DIRECT || o.points_id < 0 || o.points_id > MNN_POINTS_MIXED ||
-        o.force_m < 0 || o.chunk_images < 0 || o.gemm_lhs < 0 || o.gemm_lhs > MNN_GEMM_LHS_X || o.fused < 0 || o.fused > 2 || o.strassen < 0 || o.strassen > 1) {
+        o.force_m < 0 || o.chunk_images < 0 || o.gemm_lhs < 0 || o.gemm_lhs > MNN_GEMM_LHS_IMPLICIT || o.fused < 0 || o.fused > 2 || o.strassen < 0 || o.strassen > 1) {
         fail(MNN_EINVAL, "an option is outside its range");
         return nullptr;
     }
@@ -233,7 +238,7 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
     }
     if (o.strassen) {
         if (!strassen_applies(N, Cin, Cout, k, stride, pad, dilation, o.groups) || o.force_algo == MNN_ALGO_WINOGRAD ||
-            o.force_algo == MNN_ALGO_DIRECT || o.operand == MNN_OPERAND_FP32_REF || o.gemm_lhs == MNN_GEMM_LHS_X) {
+            o.force_algo == MNN_ALGO_DIRECT || o.operand == MNN_OPERAND_FP32_REF || o.gemm_lhs == MNN_GEMM_LHS_X || o.gemm_lhs == MNN_GEMM_LHS_IMPLICIT) {
             fail(MNN_EUNSUPPORTED, "Strassen needs a 1x1 stride-1 unpadded ungrouped layer with even N, Cin and Cout on the GEMM scheme");
             return nullptr;
         }
@@ -444,6 +449,11 @@ static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
     if (p->strassen)
         return umma_contract_setup(&p->uc, p->store_mode, 7, p->s.Cout / 2, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
                                    v_lo(p), why);
+    if (p->gemm_implicit) {
+        const LayerShape& s = p->s;
+        GatherGeom g = {s.N, s.Cin, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, p->cin_pad};
+        return implicit_gemm_setup(&p->ig, g, s.Cout, u_hi(p), why);
+    }
     if (p->gemm_x) return umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), why);
     return umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
                                v_lo(p), why);
@@ -515,7 +525,7 @@ static int check_run_args(mnn_conv_plan_t p, const float* x, const float* w, con
     if ((mask & ~(unsigned)MNN_STAGE_ALL) || mask == 0) return fail(MNN_EINVAL, "bad stage mask");
     if (p->workspace_bytes > 0 && !p->ws) return fail(MNN_EWORKSPACE, "call mnn_conv_set_workspace first");
     const bool direct = p->d.algo == MNN_ALGO_DIRECT;
-    const bool one_kernel = p->gemm_x || p->fused;       // x in, y out in the contraction stage
+    const bool one_kernel = p->gemm_x || p->gemm_implicit || p->fused;       // x in, y out in the contraction stage
     const bool need_x = direct || (!one_kernel && (mask & MNN_STAGE_INPUT)) || (one_kernel && (mask & MNN_STAGE_CONTRACT));
     const bool need_w = direct || (mask & MNN_STAGE_WEIGHT);
     const bool need_y = direct || (!p->fused && (mask & MNN_STAGE_OUTPUT)) ||
@@ -560,7 +570,9 @@ static int do_weights(mnn_conv_plan_t p, const float* w, cudaStream_t st)
 {
     cudaError_t e;
     LaunchTimer lt(p, st, 0);
-    if (p->rect)
+    if (p->gemm_implicit)
+        e = launch_implicit_weights(w, u_hi(p), p->s.Cout, p->s.Cin, p->s.k, p->cin_pad, st);
+    else if (p->rect)
         e = launch_rect_weights(w, u_hi(p), u_lo(p), rect_geom(p), p->store_mode, p->mats, st);
     else if (p->strassen)
         e = launch_strassen_weights(w, u_hi(p), u_lo(p), strassen_geom(p), p->store_mode, st);
@@ -660,7 +672,7 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
     }
     if (d.algo == MNN_ALGO_GEMM) {
         const long long T = (long long)s.N * s.OH * s.OW;
-        if ((mask & MNN_STAGE_INPUT) && !p->gemm_x) {
+        if ((mask & MNN_STAGE_INPUT) && !p->gemm_x && !p->gemm_implicit) {
             GatherGeom g = {s.N, s.Cin, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, p->cin_pad};
             LaunchTimer lt(p, st, 1);
             e = launch_gather(x, v_hi(p), v_lo(p), g, p->store_mode, st);
@@ -672,7 +684,10 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
             if (reference)
                 e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, 1, s.Cout, T, p->cin_pad,
                                               (long long)s.Cout * p->cin_pad, T * p->cin_pad, epi, st);
-            else if (p->gemm_x)
+            else if (p->gemm_implicit) {
+                GatherGeom g = {s.N, s.Cin, s.H, s.W, s.OH, s.OW, s.k, s.stride, s.pad, s.dil, p->cin_pad};
+                e = launch_implicit_gemm(p->ig, x, bias, y, g, s.relu, status_word(p), st);
+            } else if (p->gemm_x)
                 e = launch_contract_umma_x(p->uc, x, epi, status_word(p), st);
             else
                 e = launch_contract_umma(p->uc, T, epi, status_word(p), st);

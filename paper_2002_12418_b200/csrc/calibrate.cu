@@ -11,6 +11,7 @@
 
 #include "../../include/mnn_conv.h"
 #include "generator.h"
+#include "implicit_gemm.h"
 #include "contract_umma.h"
 #include "kernels.h"
 #include "planner.h"
@@ -288,6 +289,31 @@ extern "C" int mnn_calibrate(int device, void* stream, long long consts[MNN_N_CO
                 if (epi_ms < block_ms * 0.25) epi_ms = block_ms * 0.25;
                 cal.c[12] = to_ll(epi_ms * 1e9);
             }
+        }
+    }
+
+    // implicit GEMM: pace of the producer warps' gather.  3x3 stride 2, 64 -> 64 channels, 56 x 56, 4 images: 25
+    // work items of 18 blocks of 32 patch elements each, one item per SM, so the run is launch + 18 blocks + drain
+    {
+        GatherGeom g = {4, 64, 56, 56, 28, 28, 3, 2, 1, 1, 576};
+        int* status = reinterpret_cast<int*>(buf);
+        float* x = reinterpret_cast<float*>(buf + 1024);
+        float* U = x + (size_t)4 * 64 * 56 * 56;
+        float* y = U + (size_t)64 * 576;
+        cudaMemsetAsync(buf, 0, 1024, st);
+        ImplicitGemm ig;
+        const char* why = "";
+        if (implicit_gemm_setup(&ig, g, 64, U, &why) == cudaSuccess) {
+            for (int i = 0; i < 3; ++i) launch_implicit_gemm(ig, x, nullptr, y, g, 0, status, st);
+            tm.start();
+            const int reps = 20;
+            for (int i = 0; i < reps; ++i) launch_implicit_gemm(ig, x, nullptr, y, g, 0, status, st);
+            ms = tm.stop() / reps;
+            int code = 0;
+            cudaMemcpy(&code, status, sizeof(int), cudaMemcpyDeviceToHost);
+            double t = ms - (double)cal.c[5] * 1e-9;
+            if (t < ms * 0.25) t = ms * 0.25;
+            if (code == 0 && ms > 0.0) cal.c[13] = to_ll(t * 1e15 / (18.0 * 128 * 32));
         }
     }
 

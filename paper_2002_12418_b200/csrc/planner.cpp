@@ -56,6 +56,7 @@ Calibration default_calibration()
     c.c[10] = 23000000;   // as per byte of U delivered to one SM by the fused kernel's weight stream (~43 GB/s per SM)
     c.c[11] = 6000000;    // ps per 32-channel block of a fused work item (64 MMAs of 128 x 32 x 8 at ~90 ns each)
     c.c[12] = 4300000;    // ps of epilogue per fused work item
+    c.c[13] = 400000000;  // as per patch element gathered by the implicit GEMM's producer warps, per SM (~1.6 us per 128 x 32 tile)
     return c;
 }
 
@@ -343,8 +344,11 @@ bool gemm_reads_x(const LayerShape& s, int operand, int passes)
 
 namespace {
 
-uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibration& cal)
+// lhs: MNN_GEMM_LHS_PATCHES (gather kernel + GEMM), MNN_GEMM_LHS_X (the GEMM reads x itself) or
+// MNN_GEMM_LHS_IMPLICIT (producer warps gather the patches inside the GEMM kernel)
+uint64_t gemm_cost(const LayerShape& s, int operand, int lhs, const Calibration& cal)
 {
+    const bool lhs_x = lhs == MNN_GEMM_LHS_X;
     const uint64_t b = operand_bytes(operand);
     const uint64_t Kp = round_up((uint64_t)s.Cin * s.k * s.k, 8);
     const uint64_t T = (uint64_t)s.N * s.OH * s.OW;
@@ -373,6 +377,19 @@ uint64_t gemm_cost(const LayerShape& s, int operand, bool lhs_x, const Calibrati
     // (two accumulators), with about half a microsecond of hand-over per item; the last drain is exposed
     const uint64_t drain_ps = 128ull * bn * 4 * 45;
     const uint64_t loop_ps = k_blocks * (deliver_ps > mma_ps ? deliver_ps : mma_ps);
+    if (lhs == MNN_GEMM_LHS_IMPLICIT) {
+        // only the weight tile is delivered; the producers' gather of 128 x 32 patch elements paces a block too
+        const uint64_t deliver_b = (uint64_t)bn * 128 * 16;
+        // (consts[13] is measured on the tap-major gather, Cin a multiple of 32; the element-wise gather of other
+        // channel counts takes about twice as long)
+        const uint64_t gather_ps = saturate((u128)128 * 32 * (uint64_t)cal.c[13] * (s.Cin % 32 == 0 ? 1u : 2u) / 1000000u);
+        uint64_t block_ps = deliver_b > mma_ps ? deliver_b : mma_ps;
+        if (gather_ps > block_ps) block_ps = gather_ps;
+        const uint64_t loop_i = k_blocks * block_ps;
+        const uint64_t item_i = loop_i > drain_ps + 500000 ? loop_i : drain_ps + 500000;
+        const u128 serial_i = ((u128)rounds * item_i + drain_ps) * 1000000u;
+        return kernel_ps((u128)(x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_i, 0, cal);
+    }
     const uint64_t item_ps = loop_ps > drain_ps + 500000 ? loop_ps : drain_ps + 500000;
     const u128 serial_as = ((u128)rounds * item_ps + drain_ps) * 1000000u;
     if (lhs_x) return kernel_ps((u128)(x_bytes + u_bytes + y_bytes) * (uint64_t)cal.c[0], serial_as, 0, cal);
@@ -527,14 +544,29 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
             if ((uint64_t)ppm > gate_ppm && !(o.operand != 0 && o.force_algo == MNN_ALGO_GEMM)) continue;
             // left operand: the patch matrix, or x itself where that applies (whichever is cheaper)
             const bool x_ok = gemm_reads_x(s, c.operand, c.passes);
+            const bool implicit_ok = c.operand == MNN_OPERAND_TF32 && c.passes == 1;
             if (o.gemm_lhs == MNN_GEMM_LHS_X && !x_ok) continue;
-            const uint64_t cost_patches = gemm_cost(s, c.operand, false, cal);
-            const uint64_t cost_x = x_ok ? gemm_cost(s, c.operand, true, cal) : MNN_COST_INADMISSIBLE;
-            const bool take_x = o.gemm_lhs == MNN_GEMM_LHS_X || (o.gemm_lhs == MNN_GEMM_LHS_AUTO && x_ok && cost_x < cost_patches);
+            if (o.gemm_lhs == MNN_GEMM_LHS_IMPLICIT && !implicit_ok) continue;
+            const uint64_t cost_patches = gemm_cost(s, c.operand, MNN_GEMM_LHS_PATCHES, cal);
+            const uint64_t cost_x = x_ok ? gemm_cost(s, c.operand, MNN_GEMM_LHS_X, cal) : MNN_COST_INADMISSIBLE;
+            const uint64_t cost_i = implicit_ok ? gemm_cost(s, c.operand, MNN_GEMM_LHS_IMPLICIT, cal) : MNN_COST_INADMISSIBLE;
+            // left operand: as asked for, else the cheapest that applies (patch matrix, x itself, implicit gather;
+            // earlier in this order on ties; the implicit gather only once its rate constant is known)
+            int lhs = o.gemm_lhs;
+            if (lhs == MNN_GEMM_LHS_AUTO) {
+                lhs = MNN_GEMM_LHS_PATCHES;
+                uint64_t best_lhs = cost_patches;
+                if (x_ok && cost_x < best_lhs) {
+                    lhs = MNN_GEMM_LHS_X;
+                    best_lhs = cost_x;
+                }
+                if (implicit_ok && cal.c[13] > 0 && cost_i < best_lhs) lhs = MNN_GEMM_LHS_IMPLICIT;
+            }
+            const bool take_x = lhs == MNN_GEMM_LHS_X;
             if (take_x && ppm < kGemmLhsXErrorPpm) ppm = kGemmLhsXErrorPpm;
-            lhs_of[i] = take_x ? MNN_GEMM_LHS_X : MNN_GEMM_LHS_PATCHES;
+            lhs_of[i] = lhs;
             ppm_of[i] = ppm;
-            d->cost_ps[i] = take_x ? cost_x : cost_patches;
+            d->cost_ps[i] = lhs == MNN_GEMM_LHS_X ? cost_x : (lhs == MNN_GEMM_LHS_IMPLICIT ? cost_i : cost_patches);
             continue;
         }
         // Winograd

@@ -20,7 +20,7 @@ from . import binding as B
 STAGES = {"weight": B.STAGE_WEIGHT, "input": B.STAGE_INPUT, "contract": B.STAGE_CONTRACT, "output": B.STAGE_OUTPUT,
           "all": B.STAGE_INPUT | B.STAGE_CONTRACT | B.STAGE_OUTPUT}
 OPERANDS = {"auto": B.OPERAND_AUTO, "tf32": B.OPERAND_TF32, "bf16": B.OPERAND_BF16, "fp32ref": B.OPERAND_FP32_REF}
-LHS = {"auto": B.GEMM_LHS_AUTO, "patches": B.GEMM_LHS_PATCHES, "x": B.GEMM_LHS_X}
+LHS = {"auto": B.GEMM_LHS_AUTO, "patches": B.GEMM_LHS_PATCHES, "x": B.GEMM_LHS_X, "implicit": B.GEMM_LHS_IMPLICIT}
 ALGOS = {"auto": B.ALGO_AUTO, "winograd": B.ALGO_WINOGRAD, "gemm": B.ALGO_GEMM, "direct": B.ALGO_DIRECT}
 
 
@@ -49,7 +49,7 @@ def stage_work(info, N, Cin, Cout, H, W, k, groups):
     elif info.algo == B.ALGO_GEMM:
         K, T = Cin * k * k, N * info.OH * info.OW
         v = b_el * T * K
-        if info.gemm_lhs == B.GEMM_LHS_X:
+        if info.gemm_lhs in (B.GEMM_LHS_X, B.GEMM_LHS_IMPLICIT):
             v = x_bytes                    # the contraction reads x itself
         else:
             out["input"] = (x_bytes + v, 0)

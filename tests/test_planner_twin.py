@@ -83,7 +83,7 @@ def restore_calibration():
     B.mnn_set_calibration(before)
 
 
-PERTURBED = [211000, 61000, 2500, 900, 35000, 5100000, 40 << 20, 132, 480000, 45000, 15000, 900000, 2500000, 0, 0, 0]
+PERTURBED = [211000, 61000, 2500, 900, 35000, 5100000, 40 << 20, 132, 480000, 45000, 15000, 900000, 2500000, 90000000, 0, 0]
 
 
 @pytest.mark.parametrize("record", ["builtin", "perturbed"])
@@ -117,8 +117,16 @@ def test_forced_options_match_the_twin(restore_calibration):
     for okw, tkw in cases:
         compare(l, okw, tkw, cal)
     pw = W.config3(64)[2]
-    for lhs in (B.GEMM_LHS_PATCHES, B.GEMM_LHS_X):
+    for lhs in (B.GEMM_LHS_PATCHES, B.GEMM_LHS_X, B.GEMM_LHS_IMPLICIT):
         compare(pw, dict(gemm_lhs=lhs), dict(gemm_lhs=lhs), cal)
+    s2 = W.config2(32)[5]                                   # 3x3 stride 2: patches or the implicit gather
+    for lhs in (B.GEMM_LHS_PATCHES, B.GEMM_LHS_IMPLICIT):
+        compare(s2, dict(force_algo=B.ALGO_GEMM, gemm_lhs=lhs), dict(force_algo=T.ALGO_GEMM, gemm_lhs=lhs), cal)
+    fast = list(cal)
+    fast[13] = 1000                                         # a gather that costs nothing: the planner takes it by itself
+    B.mnn_set_calibration(fast)
+    info = compare(s2, dict(force_algo=B.ALGO_GEMM), dict(force_algo=T.ALGO_GEMM), fast)
+    assert info.gemm_lhs == B.GEMM_LHS_IMPLICIT
 
 
 def test_fused_candidate_disappears_without_its_constants(restore_calibration):
