@@ -19,8 +19,9 @@ def test_mobilenet_stack_layout_shares_the_transient_part():
     assert info.workspace_bytes == info.persistent_bytes + info.transient_bytes + 2 * info.activation_bytes
     largest_act = max(4 * 64 * l.Cout * l.OH * l.OW for l in layers[:-1])
     assert largest_act <= info.activation_bytes < largest_act + 1024
-    # sharing pays: the per-layer workspaces added up are larger than persistent + transient
-    assert info.persistent_bytes + info.transient_bytes < info.sum_of_layer_workspaces
+    # sharing never costs: persistent + one transient part is at most the per-layer workspaces added up (equal when
+    # no layer of the stack needs a transient part, e.g. when every GEMM reads x itself or gathers implicitly)
+    assert info.persistent_bytes + info.transient_bytes <= info.sum_of_layer_workspaces
     B.mnn_net_destroy(net)
 
 
