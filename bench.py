@@ -544,7 +544,7 @@ def gpu_rank_main(args):
                 "config": {"workload": args.workload, "layers": len(layers), "batch_per_gpu": layers[0].N,
                            "l2": "flushed before every step (256 MB write)", "weights": "pre-transformed",
                            "launch": "CUDA graph replay per step" if args.launch == "graph" else "C-ABI calls on the stream",
-                           "accuracy_class": args.precision, "planner_calibration": calibration[:13],
+                           "accuracy_class": args.precision, "planner_calibration": calibration[:14],
                            "calibration_source": args.calibration, "plans": main_res["plans"]},
                 "clocks": main_res["clocks"], "roofline": main_res["roofline"],
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

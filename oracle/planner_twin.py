@@ -342,7 +342,8 @@ def plan(L: Layer, o: Options, c, ppm) -> Choice:
                 lhs = LHS_PATCHES
                 if x_ok and costs[LHS_X] < costs[lhs]:
                     lhs = LHS_X
-                if implicit_ok and c[13] > 0 and costs[LHS_IMPLICIT] < costs[lhs]:
+                # (plain pointwise layers keep the tuned paths: measured, the implicit gather never beat them there)
+                if implicit_ok and not (L.k == 1 and L.stride == 1) and c[13] > 0 and costs[LHS_IMPLICIT] < costs[lhs]:
                     lhs = LHS_IMPLICIT
             if lhs == LHS_X:
                 p = max(p, LHS_X_ERROR_PPM)

@@ -560,7 +560,9 @@ int plan_layer(const LayerShape& s, const mnn_conv_opts& o, const Calibration& c
                     lhs = MNN_GEMM_LHS_X;
                     best_lhs = cost_x;
                 }
-                if (implicit_ok && cal.c[13] > 0 && cost_i < best_lhs) lhs = MNN_GEMM_LHS_IMPLICIT;
+                // (plain pointwise layers keep the tuned paths: measured, the implicit gather never beat them there)
+                const bool pointwise = s.k == 1 && s.stride == 1;
+                if (implicit_ok && !pointwise && cal.c[13] > 0 && cost_i < best_lhs) lhs = MNN_GEMM_LHS_IMPLICIT;
             }
             const bool take_x = lhs == MNN_GEMM_LHS_X;
             if (take_x && ppm < kGemmLhsXErrorPpm) ppm = kGemmLhsXErrorPpm;
