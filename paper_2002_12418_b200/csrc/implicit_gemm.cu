@@ -116,7 +116,7 @@ implicit_gemm_kernel(const __grid_constant__ CUtensorMap map_u, IgParams p)
             for (long long item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const int nb = (int)(item / p.n_tile_blocks);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, abortp)) {
+                    if (!ptx::mbar_wait_relaxed(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, abortp)) {
                         if (!*abortp) atomicCAS(p.status, 0, kErrTmaWait);
                         *abortp = 1;
                         ok = false;
@@ -181,7 +181,7 @@ implicit_gemm_kernel(const __grid_constant__ CUtensorMap map_u, IgParams p)
             const int tb = (int)(item % p.n_tile_blocks);
             const int nb = (int)(item / p.n_tile_blocks);
             int got = 1;
-            if (lane == 0) got = ptx::mbar_wait_bounded(ptx::smem_u32(&tfull_bar[acc]), acc_phase, abortp) ? 1 : 0;
+            if (lane == 0) got = ptx::mbar_wait_relaxed(ptx::smem_u32(&tfull_bar[acc]), acc_phase, abortp) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) {
                 if (lane == 0) {
@@ -345,7 +345,7 @@ implicit_gemm_kernel(const __grid_constant__ CUtensorMap map_u, IgParams p)
                 if (s + 2 < n_steps) gather(s + 2, vb);
             }
             int got = 1;
-            if (lane == 0) got = ptx::mbar_wait_bounded(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, abortp) ? 1 : 0;
+            if (lane == 0) got = ptx::mbar_wait_relaxed(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, abortp) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) {
                 if (lane == 0) {

@@ -196,7 +196,7 @@ fused_f2x2_3x3_kernel(const __grid_constant__ wino::MatBt2 Bt, MatAt4 At, FusedP
                 const int cb = item / p.n_tile_blocks;
                 const uint8_t* src = p.U + (size_t)cb * p.k_blocks * kUBlockBytes;
                 for (int c = 0; c < p.k_blocks * kGroups; ++c) {           // consecutive copies are consecutive in memory
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&u_empty[slot]), phase ^ 1u, abortp)) {
+                    if (!ptx::mbar_wait_relaxed(ptx::smem_u32(&u_empty[slot]), phase ^ 1u, abortp)) {
                         if (!*abortp) atomicCAS(p.status, 0, kErrStreamWait);
                         *abortp = 1;
                         ok = false;
@@ -281,7 +281,7 @@ fused_f2x2_3x3_kernel(const __grid_constant__ wino::MatBt2 Bt, MatAt4 At, FusedP
         for (int item = first; item < p.n_items; item += step) {
             const int cb = item / p.n_tile_blocks, tb = item - cb * p.n_tile_blocks;
             int got = 1;
-            if (lane == 0) got = ptx::mbar_wait_bounded(ptx::smem_u32(&acc_full), acc_phase, abortp) ? 1 : 0;
+            if (lane == 0) got = ptx::mbar_wait_relaxed(ptx::smem_u32(&acc_full), acc_phase, abortp) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) {
                 if (lane == 0) {
@@ -410,7 +410,7 @@ fused_f2x2_3x3_kernel(const __grid_constant__ wino::MatBt2 Bt, MatAt4 At, FusedP
             // ... and request the next one, so that its latency is covered by this step's arithmetic and stores
             if (s + 1 < n_steps) step_window(s + 1, d);
             int got = 1;
-            if (lane == 0) got = ptx::mbar_wait_bounded(ptx::smem_u32(&v_empty[buf]), v_phase ^ 1u, abortp) ? 1 : 0;
+            if (lane == 0) got = ptx::mbar_wait_relaxed(ptx::smem_u32(&v_empty[buf]), v_phase ^ 1u, abortp) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) {
                 if (lane == 0) {
