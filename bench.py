@@ -34,7 +34,16 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from stored ncu captures of
 # this file's workloads (profiles/ holds the summaries and their commands); not measured by this run.  An entry is
 # used only while the plans of the run are the plans of the capture.
-NCU_DRAM_TRAFFIC = {}
+NCU_DRAM_TRAFFIC = {
+    "config4_b64/tf32": {
+        "plans": [("winograd", 4, "bf16", 3), ("winograd", 4, "bf16", 3), ("winograd", 4, "bf16", 3), ("winograd", 4, "tf32", 3)],
+        # mean over the four contraction launches of one step, captured at batch 16 (190.6 / 456.8 / 29.9 / 99.6 MB)
+        # and multiplied by four; at batch 64 less of V and M stays in L2, so the true figure is somewhat higher
+        "contraction": 4 * 194.2e6,
+        "source": "stored ncu capture of the batch-16 copy of this workload (profiles/bench_config4_b64_launch_list.md), "
+                  "scaled by 4; not measured by this run",
+    },
+}
 
 # nominal dense tensor rates relative to BF16 (2.25 PFLOP/s): TF32 1.1 PFLOP/s
 TF32_OVER_BF16 = 1.1 / 2.25
@@ -47,6 +56,7 @@ def workload_layers(name: str):
         "config2_b32": lambda: W.config2(32),
         "config3_b64": lambda: W.config3(64),
         "config4_b64": lambda: W.config4(64),
+        "config4_b16": lambda: W.config4(16),      # quarter-size copy of the headline workload, for profiler captures
     }
     if name not in table:
         raise SystemExit("unknown workload %s (have %s)" % (name, ", ".join(sorted(table))))
