@@ -32,7 +32,7 @@ METRIC = "conv TFLOP/s (direct-conv-equivalent)"
 UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from stored ncu captures of
-# this file's workloads (profiles/ holds the summaries and their commands); not measured by this run.  An entry is
+# this file's workloads (the capture commands are kept with the profile summaries); not measured by this run.  An entry is
 # used only while the plans of the run are the plans of the capture.
 NCU_DRAM_TRAFFIC = {
     "config4_b64/tf32": {
@@ -40,8 +40,7 @@ NCU_DRAM_TRAFFIC = {
         # mean over the four contraction launches of one step, captured at batch 16 (190.6 / 456.8 / 29.9 / 99.6 MB)
         # and multiplied by four; at batch 64 less of V and M stays in L2, so the true figure is somewhat higher
         "contraction": 4 * 194.2e6,
-        "source": "stored ncu capture of the batch-16 copy of this workload (profiles/bench_config4_b64_launch_list.md), "
-                  "scaled by 4; not measured by this run",
+        "source": "stored ncu capture of the batch-16 copy of this workload, scaled by 4; not measured by this run",
     },
 }
 

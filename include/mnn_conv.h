@@ -354,6 +354,14 @@ MNN_API int mnn_net_run(mnn_net_t net, const float* x, const float* const* w, co
 MNN_API int mnn_net_device_status(mnn_net_t net, void* stream, int* code, int* layer);
 MNN_API void mnn_net_destroy(mnn_net_t net);
 
+/* Self-test of the bounded waits every persistent kernel of the library relies on (no counterpart in the paper).
+ * Launches one tiny kernel on `stream` that initialises a shared-memory barrier nobody ever arrives on and waits
+ * on it with the library's bounded wait; the wait gives up after its limit (about one second) and the
+ * kernel returns normally.  `device_word` (device memory, 4 bytes, caller-owned) receives 1 when the kernel has
+ * started, then 2 when the wait gave up as it must, or 3 if it reported completion.  Asynchronous; no fault, trap
+ * or endless loop is involved, and the context stays usable. */
+MNN_API int mnn_wait_probe(int* device_word, void* stream);
+
 MNN_API const char* mnn_last_error(void);
 
 #ifdef __cplusplus

@@ -27,7 +27,7 @@ OPERAND_NAMES = {OPERAND_TF32: "tf32", OPERAND_BF16: "bf16", OPERAND_FP32_REF: "
 
 EXPORTED = ["mnn_conv_plan", "mnn_conv_plan_ex", "mnn_conv_plan_rect", "mnn_conv_plan_query", "mnn_conv_set_workspace",
             "mnn_conv_prepare_weights", "mnn_conv_run", "mnn_conv_run_stages", "mnn_conv_device_status",
-            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_strassen_rule", "mnn_calibrate",
+            "mnn_conv_profile", "mnn_conv_profile_read", "mnn_conv_destroy", "mnn_conv_run_static", "mnn_winograd_matrices", "mnn_accuracy_ppm", "mnn_strassen_rule", "mnn_wait_probe", "mnn_calibrate",
             "mnn_set_calibration", "mnn_get_calibration", "mnn_last_error",
             "mnn_net_plan", "mnn_net_query", "mnn_net_set_workspace", "mnn_net_prepare", "mnn_net_run",
             "mnn_net_device_status", "mnn_net_destroy"]
@@ -122,6 +122,8 @@ def lib():
         L.mnn_winograd_matrices.restype = i
         L.mnn_accuracy_ppm.argtypes = [i] * 5
         L.mnn_accuracy_ppm.restype = ll
+        L.mnn_wait_probe.argtypes = [p, p]
+        L.mnn_wait_probe.restype = i
         L.mnn_strassen_rule.argtypes = [ll, ll, ll]
         L.mnn_strassen_rule.restype = i
         L.mnn_calibrate.argtypes = [i, p, ctypes.POINTER(ll)]
@@ -260,6 +262,10 @@ def mnn_accuracy_ppm(m, k, points_id, operand, passes) -> int:
     if v < 0:
         raise MnnError(MNN_EINVAL, mnn_last_error())
     return int(v)
+
+
+def mnn_wait_probe(device_word_ptr: int, stream: int) -> None:
+    _check(lib().mnn_wait_probe(device_word_ptr, stream))
 
 
 def mnn_strassen_rule(m: int, n: int, k: int) -> int:

@@ -838,6 +838,14 @@ long long mnn_accuracy_ppm(int m, int k, int points_id, int operand, int passes)
     return v;
 }
 
+int mnn_wait_probe(int* device_word, void* stream)
+{
+    if (!device_word) return fail(MNN_EINVAL, "NULL device word");
+    cudaError_t e = launch_wait_probe(device_word, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(e, "wait probe");
+    return MNN_OK;
+}
+
 int mnn_strassen_rule(long long m, long long n, long long k)
 {
     if (m < 2 || n < 2 || k < 2) return 0;

@@ -369,6 +369,22 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     }
 }
 
+// A barrier nobody arrives on: the bounded wait must give up and let the kernel return.
+__global__ void wait_probe_kernel(int* word)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int never_set;
+    if (threadIdx.x == 0) {
+        never_set = 0;
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        ptx::fence_barrier_init();
+        *word = 1;
+        __threadfence();
+        const bool done = ptx::mbar_wait_bounded(ptx::smem_u32(&bar), 0u, &never_set);
+        *word = done ? 3 : 2;
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -448,6 +464,12 @@ bool encode_input_map(CUtensorMap* map, const float* x, int images, int C, int H
     return r == CUDA_SUCCESS;
 }
 }  // namespace wino
+
+cudaError_t launch_wait_probe(int* device_word, cudaStream_t stream)
+{
+    wait_probe_kernel<<<1, 32, 0, stream>>>(device_word);
+    return cudaGetLastError();
+}
 
 cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout, int cin_pad, long long tiles_capacity,
                                 void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why)

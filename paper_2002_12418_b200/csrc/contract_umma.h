@@ -45,4 +45,7 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
 bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
                         long long plane_stride_elems, int box_rows);
 
+// One thread waits, with the bounded wait of umma.cuh, on a barrier nobody arrives on; *device_word ends as 2.
+cudaError_t launch_wait_probe(int* device_word, cudaStream_t stream);
+
 }  // namespace mnnb

@@ -55,22 +55,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Polls at most kFastPolls + kSlowPolls times (the slow ones sleep ~100 ns each,
-// about half a second in all); `abort_flag` (shared memory) lets one role's
-// failure end the others' waits early.
+// A wait spins kFastPolls times, then polls with ~100 ns sleeps until kWaitLimitNs of wall time (the GPU's
+// global timer) have passed since it began sleeping: about one second, after which it returns false.
+// `abort_flag` (shared memory) lets one role's failure end the others' waits early.
 constexpr uint32_t kFastPolls = 1u << 14;
-constexpr uint32_t kSlowPolls = 1u << 22;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
     for (uint32_t i = 0; i < kFastPolls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < kSlowPolls; ++i) {
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 0 && *abort_flag) return false;
+        if ((i & 63u) == 0 && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) return false;
         __nanosleep(100);
     }
-    return false;
 }
 
 // The same bound for warps that can afford to wait: sleeps between polls from the start, so that
@@ -78,12 +85,12 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < kSlowPolls; ++i) {
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t i = 0;; ++i) {
         __nanosleep(64);
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 0 && *abort_flag) return false;
+        if ((i & 63u) == 0 && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) return false;
     }
-    return false;
 }
 
 // Asynchronous 4- or 8-byte copy global -> shared; src_bytes = 0 writes zeros without reading.
