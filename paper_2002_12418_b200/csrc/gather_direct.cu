@@ -366,6 +366,197 @@ __global__ void __launch_bounds__(kStemThreads) direct_stem_kernel(const float* 
     }
 }
 
+// The same layer with its shape fixed at compile time (dilation 1): all CIN * K * K input values of a thread's
+// PIX output pixels are requested before the first is used, and the multiply-adds run as packed pairs of fp32
+// lanes (__ffma2_rn: two IEEE fused multiply-adds per instruction, the results of the scalar kernel bit for
+// bit), with one shared-memory weight fetch serving all PIX pixels.
+template <int CIN, int K, int STRIDE, int PIX>
+__global__ void __launch_bounds__(kStemThreads) direct_stem_fixed_kernel(const float* __restrict__ x, const float* __restrict__ w,
+                                                                         const float* __restrict__ bias, float* __restrict__ y,
+                                                                         DirectGeom g, int co_pad)
+{
+    constexpr int TAPS = CIN * K * K;
+    extern __shared__ __align__(16) float s_w[];              // [TAPS][co_pad]
+    for (int i = threadIdx.x; i < TAPS * co_pad; i += kStemThreads) {
+        const int tap = i / co_pad, co = i - tap * co_pad;
+        s_w[i] = co < g.Cout ? __ldg(w + (size_t)co * TAPS + tap) : 0.0f;
+    }
+    __syncthreads();
+    const int ohw = g.OH * g.OW;
+    const int n = blockIdx.y;
+    const int pix0 = blockIdx.x * (kStemThreads * PIX) + threadIdx.x;
+    const float* xn = x + (size_t)n * CIN * g.H * g.W;
+    float v[PIX][TAPS];
+#pragma unroll
+    for (int p = 0; p < PIX; ++p) {
+        const int pix = pix0 + p * kStemThreads;
+        const bool live = pix < ohw;
+        const int oh = pix / g.OW, ow = pix - oh * g.OW;
+        const int ih0 = oh * STRIDE - g.pad, iw0 = ow * STRIDE - g.pad;
+#pragma unroll
+        for (int ci = 0; ci < CIN; ++ci)
+#pragma unroll
+            for (int a = 0; a < K; ++a)
+#pragma unroll
+                for (int b = 0; b < K; ++b) {
+                    const int ih = ih0 + a, iw = iw0 + b;
+                    const bool ok = live && ih >= 0 && ih < g.H && iw >= 0 && iw < g.W;
+                    v[p][(ci * K + a) * K + b] = ok ? __ldg(xn + ((size_t)ci * g.H + ih) * g.W + iw) : 0.0f;
+                }
+    }
+    for (int c0 = 0; c0 < g.Cout; c0 += kStemCoChunk) {
+        float2 acc[PIX][kStemCoChunk / 2];
+#pragma unroll
+        for (int j = 0; j < kStemCoChunk / 2; ++j) {
+            const float b0 = (bias && c0 + 2 * j < g.Cout) ? __ldg(bias + c0 + 2 * j) : 0.0f;
+            const float b1 = (bias && c0 + 2 * j + 1 < g.Cout) ? __ldg(bias + c0 + 2 * j + 1) : 0.0f;
+#pragma unroll
+            for (int p = 0; p < PIX; ++p) acc[p][j] = make_float2(b0, b1);
+        }
+#pragma unroll
+        for (int tap = 0; tap < TAPS; ++tap) {
+            const float4* wp = reinterpret_cast<const float4*>(s_w + (size_t)tap * co_pad + c0);
+            float2 vv[PIX];
+#pragma unroll
+            for (int p = 0; p < PIX; ++p) vv[p] = make_float2(v[p][tap], v[p][tap]);
+#pragma unroll
+            for (int q = 0; q < kStemCoChunk / 4; ++q) {
+                const float4 w4 = wp[q];
+#pragma unroll
+                for (int p = 0; p < PIX; ++p) {
+                    acc[p][2 * q] = __ffma2_rn(make_float2(w4.x, w4.y), vv[p], acc[p][2 * q]);
+                    acc[p][2 * q + 1] = __ffma2_rn(make_float2(w4.z, w4.w), vv[p], acc[p][2 * q + 1]);
+                }
+            }
+        }
+        const bool full = c0 + kStemCoChunk <= g.Cout;
+#pragma unroll
+        for (int p = 0; p < PIX; ++p) {
+            const int pix = pix0 + p * kStemThreads;
+            if (pix >= ohw) continue;
+            float* yp = y + ((size_t)n * g.Cout + c0) * ohw + pix;
+#pragma unroll
+            for (int j = 0; j < kStemCoChunk / 2; ++j) {
+                float lo = acc[p][j].x, hi = acc[p][j].y;
+                if (g.relu) { lo = fmaxf(lo, 0.0f); hi = fmaxf(hi, 0.0f); }
+                if (full || c0 + 2 * j < g.Cout) yp[(size_t)(2 * j) * ohw] = lo;
+                if (full || c0 + 2 * j + 1 < g.Cout) yp[(size_t)(2 * j + 1) * ohw] = hi;
+            }
+        }
+    }
+}
+
+// 3 -> Cout, 3x3, stride 2, padding 1 on planes with H even and W a multiple of 4 (the first layer of the
+// ImageNet networks).  A thread owns a block of ROWS x 2 output pixels (ROWS = 2 when H is a multiple of 4):
+// its (2 ROWS + 1) x 5 x 3 input values come from two aligned float2 loads and one scalar load per row, the two
+// results of a channel and row leave as one float2 store, and only the row above the plane and the column
+// left of it can fall outside.  One 16-byte weight fetch from shared memory feeds 2 ROWS packed multiply-adds
+// (__ffma2_rn: two IEEE fused multiply-adds per instruction, bit for bit the scalar result).  Blocks walk
+// over (image, group of 128 pixel blocks) units and stage the weights once.
+constexpr int kPairCoChunk = 16;   // output channels per sweep over the 27 taps
+
+template <bool RELU, int ROWS>
+__global__ void __launch_bounds__(kStemThreads, ROWS == 1 ? 5 : 3)
+direct_stem_s2_pair_kernel(const float* __restrict__ x, const float* __restrict__ w, const float* __restrict__ bias,
+                           float* __restrict__ y, DirectGeom g, int co_pad, int groups, int n_units)
+{
+    constexpr int CIN = 3, K = 3, TAPS = CIN * K * K, NR = 2 * ROWS + 1, PIX = 2 * ROWS;
+    extern __shared__ __align__(16) float s_w[];              // [TAPS][co_pad]
+    for (int i = threadIdx.x; i < TAPS * co_pad; i += kStemThreads) {
+        const int tap = i / co_pad, co = i - tap * co_pad;
+        s_w[i] = co < g.Cout ? __ldg(w + (size_t)co * TAPS + tap) : 0.0f;
+    }
+    __syncthreads();
+    const int ohw = g.OH * g.OW, half_w = g.OW >> 1, per_image = (g.OH / ROWS) * half_w;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int n = unit / groups;
+        const int pp = (unit - n * groups) * kStemThreads + threadIdx.x;
+        if (pp >= per_image) continue;
+        const int obr = pp / half_w;
+        const int oh = obr * ROWS, ow = 2 * (pp - obr * half_w);
+        const float* xn = x + (size_t)n * CIN * g.H * g.W + 2 * ow;
+        float c[CIN][NR][5];
+#pragma unroll
+        for (int ci = 0; ci < CIN; ++ci)
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+                const int ih = 2 * oh - 1 + r;
+                const bool row_ok = ih >= 0 && ih < g.H;
+                const float* row = xn + ((size_t)ci * g.H + (row_ok ? ih : 0)) * g.W;
+                const float2 m0 = __ldg(reinterpret_cast<const float2*>(row));
+                const float2 m1 = __ldg(reinterpret_cast<const float2*>(row + 2));
+                const float left = ow > 0 ? __ldg(row - 1) : 0.0f;
+                c[ci][r][0] = row_ok ? left : 0.0f;
+                c[ci][r][1] = row_ok ? m0.x : 0.0f;
+                c[ci][r][2] = row_ok ? m0.y : 0.0f;
+                c[ci][r][3] = row_ok ? m1.x : 0.0f;
+                c[ci][r][4] = row_ok ? m1.y : 0.0f;
+            }
+        for (int c0 = 0; c0 < g.Cout; c0 += kPairCoChunk) {
+            float2 acc[PIX][kPairCoChunk / 2];                 // pixel = 2 * row + column
+#pragma unroll
+            for (int j = 0; j < kPairCoChunk / 2; ++j) {
+                const float b0 = (bias && c0 + 2 * j < g.Cout) ? __ldg(bias + c0 + 2 * j) : 0.0f;
+                const float b1 = (bias && c0 + 2 * j + 1 < g.Cout) ? __ldg(bias + c0 + 2 * j + 1) : 0.0f;
+#pragma unroll
+                for (int p = 0; p < PIX; ++p) acc[p][j] = make_float2(b0, b1);
+            }
+            // the weights of tap t + 1 are fetched while tap t is multiplied
+            const float4* wbase = reinterpret_cast<const float4*>(s_w + c0);
+            const int wstep = co_pad >> 2;
+            float4 wn[kPairCoChunk / 4];
+#pragma unroll
+            for (int q = 0; q < kPairCoChunk / 4; ++q) wn[q] = wbase[q];
+#pragma unroll
+            for (int ci = 0; ci < CIN; ++ci)
+#pragma unroll
+                for (int a = 0; a < K; ++a)
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const int tap = (ci * K + a) * K + b;
+                        float4 wc[kPairCoChunk / 4];
+#pragma unroll
+                        for (int q = 0; q < kPairCoChunk / 4; ++q) wc[q] = wn[q];
+                        if (tap + 1 < TAPS) {
+#pragma unroll
+                            for (int q = 0; q < kPairCoChunk / 4; ++q) wn[q] = wbase[(tap + 1) * wstep + q];
+                        }
+                        float2 v[PIX];
+#pragma unroll
+                        for (int p = 0; p < PIX; ++p) {
+                            const float e = c[ci][2 * (p >> 1) + a][b + 2 * (p & 1)];
+                            v[p] = make_float2(e, e);
+                        }
+#pragma unroll
+                        for (int q = 0; q < kPairCoChunk / 4; ++q) {
+                            const float4 w4 = wc[q];
+#pragma unroll
+                            for (int p = 0; p < PIX; ++p) {
+                                acc[p][2 * q] = __ffma2_rn(make_float2(w4.x, w4.y), v[p], acc[p][2 * q]);
+                                acc[p][2 * q + 1] = __ffma2_rn(make_float2(w4.z, w4.w), v[p], acc[p][2 * q + 1]);
+                            }
+                        }
+                    }
+            const bool full = c0 + kPairCoChunk <= g.Cout;
+#pragma unroll
+            for (int rr = 0; rr < ROWS; ++rr) {
+                float* yp = y + ((size_t)n * g.Cout + c0) * ohw + (size_t)(oh + rr) * g.OW + ow;
+#pragma unroll
+                for (int j = 0; j < kPairCoChunk / 2; ++j) {
+                    float2 e = make_float2(acc[2 * rr][j].x, acc[2 * rr + 1][j].x);
+                    float2 o = make_float2(acc[2 * rr][j].y, acc[2 * rr + 1][j].y);
+                    if (RELU) {
+                        e.x = fmaxf(e.x, 0.0f); e.y = fmaxf(e.y, 0.0f);
+                        o.x = fmaxf(o.x, 0.0f); o.y = fmaxf(o.y, 0.0f);
+                    }
+                    if (full || c0 + 2 * j < g.Cout) *reinterpret_cast<float2*>(yp + (size_t)(2 * j) * ohw) = e;
+                    if (full || c0 + 2 * j + 1 < g.Cout) *reinterpret_cast<float2*>(yp + (size_t)(2 * j + 1) * ohw) = o;
+                }
+            }
+        }
+    }
+}
+
 // Depthwise 3x3 (groups = C, dilation 1, padding 1, stride 1 or 2): one warp sweeps a strip of one channel
 // plane downwards over a band of output rows.  A lane holds its column of the three input rows that an output
 // row needs; horizontal neighbours come from warp shuffles, so every input element is loaded once per strip
@@ -724,6 +915,29 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
         if (smem > 48 * 1024) {
             cudaError_t e = cudaFuncSetAttribute(direct_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
+        }
+        if (g.Cin == 3 && g.k == 3 && g.dil == 1 && g.stride == 2 && g.pad == 1 && g.H % 2 == 0 && g.W % 4 == 0 &&
+            smem <= 48 * 1024 && reinterpret_cast<uintptr_t>(x) % 8 == 0 && reinterpret_cast<uintptr_t>(y) % 8 == 0) {
+            const int rows = g.H % 4 == 0 ? 2 : 1;
+            const int per_image = (g.OH / rows) * (g.OW / 2);
+            const int groups = (per_image + kStemThreads - 1) / kStemThreads;
+            const long long units = (long long)g.N * groups;
+            if (units <= 2147483647ll) {
+                const int resident = 148 * (rows == 1 ? 5 : 3);
+                const unsigned blocks = (unsigned)(units < resident ? units : resident);
+#define MNNB_STEM_PAIR(RELU, ROWS) direct_stem_s2_pair_kernel<RELU, ROWS><<<blocks, kStemThreads, smem, stream>>>(x, w, bias, y, g, co_pad, groups, (int)units)
+                if (rows == 2) { if (g.relu) MNNB_STEM_PAIR(true, 2); else MNNB_STEM_PAIR(false, 2); }
+                else { if (g.relu) MNNB_STEM_PAIR(true, 1); else MNNB_STEM_PAIR(false, 1); }
+#undef MNNB_STEM_PAIR
+                return cudaGetLastError();
+            }
+        }
+        if (g.Cin == 3 && g.k == 3 && g.dil == 1 && (g.stride == 1 || g.stride == 2) && smem <= 48 * 1024) {
+            constexpr int kPix = 2;
+            const dim3 grid2((unsigned)((g.OH * g.OW + kStemThreads * kPix - 1) / (kStemThreads * kPix)), (unsigned)g.N);
+            if (g.stride == 2) direct_stem_fixed_kernel<3, 3, 2, kPix><<<grid2, kStemThreads, smem, stream>>>(x, w, bias, y, g, co_pad);
+            else direct_stem_fixed_kernel<3, 3, 1, kPix><<<grid2, kStemThreads, smem, stream>>>(x, w, bias, y, g, co_pad);
+            return cudaGetLastError();
         }
         const dim3 grid((unsigned)((g.OH * g.OW + kStemThreads - 1) / kStemThreads), (unsigned)g.N);
         direct_stem_kernel<<<grid, kStemThreads, smem, stream>>>(x, w, bias, y, g, co_pad);

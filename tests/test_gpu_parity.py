@@ -388,13 +388,27 @@ def test_depthwise_even_widths(torch, C, H, W_, N, stride):
 
 @pytest.mark.parametrize("Cin,Cout,H,k,stride,pad,dil,groups", [
     (3, 32, 32, 3, 2, 1, 1, 1), (3, 16, 30, 7, 2, 3, 1, 1), (6, 6, 9, 3, 1, 1, 2, 6), (5, 7, 8, 2, 1, 0, 1, 1),
-    (4, 4, 6, 5, 3, 2, 1, 4)])
+    (4, 4, 6, 5, 3, 2, 1, 4), (3, 40, 37, 3, 2, 1, 1, 1), (3, 24, 19, 3, 1, 1, 1, 1), (3, 33, 50, 3, 2, 0, 1, 1)])
 def test_generic_direct(torch, Cin, Cout, H, k, stride, pad, dil, groups):
     layer = W.ConvLayer("t", 2, Cin, Cout, H, H, k, stride, pad, dil, groups=groups, relu=True, seed=k)
     x, w, b = W.make_inputs(layer)
     got, info, _ = run_layer(torch, layer, opts_for(layer, force_algo=B.ALGO_DIRECT), (x, w, b))
     assert info.algo == B.ALGO_DIRECT
     assert rel_l2(got, oracle(layer, x, w, b)) < 1e-6
+
+
+@pytest.mark.parametrize("Cout,H,Wd,relu", [(70, 30, 44, False), (32, 64, 64, True), (5, 2, 4, True), (21, 8, 12, False), (48, 100, 36, True)])
+def test_stem_pixel_pairs(torch, Cout, H, Wd, relu):
+    """3 -> Cout 3x3 stride 2 padding 1 with H even and W a multiple of 4: the kernel that owns two adjacent
+    output pixels per thread; integers make the comparison exact, floats check the accumulation."""
+    layer = W.ConvLayer("t", 3, 3, Cout, H, Wd, 3, 2, 1, 1, relu=relu, seed=Cout)
+    x, w, b = W.make_inputs(layer)
+    got, info, _ = run_layer(torch, layer, opts_for(layer, force_algo=B.ALGO_DIRECT), (x, w, b))
+    assert info.algo == B.ALGO_DIRECT
+    assert rel_l2(got, oracle(layer, x, w, b)) < 1e-6
+    xi, wi, bi = W.integer_inputs(layer, -3, 3)
+    goti, _, _ = run_layer(torch, layer, opts_for(layer, force_algo=B.ALGO_DIRECT), (xi, wi, bi))
+    assert np.array_equal(goti.astype(np.float64), oracle(layer, xi, wi, bi))
 
 
 def test_integer_direct_and_winograd_exact(torch):
