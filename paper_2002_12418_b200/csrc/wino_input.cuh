@@ -78,24 +78,32 @@ __device__ __forceinline__ float2 v_sub(float2 a, float2 b) { return __ffma2_rn(
 __device__ __forceinline__ float v_make(float a, float, float) { return a; }
 __device__ __forceinline__ float2 v_make(float a, float b, float2) { return make_float2(a, b); }
 
-// One 1-D pass o = B^T d.  SYM: the symmetric-point structure described above.
-template <int ALPHA, bool SYM, typename T>
+// One 1-D pass o = B^T d, outputs LO .. HI - 1 only (the others are left untouched).  SYM: the
+// symmetric-point structure described above; LO and HI are then 0 / ALPHA or odd, so that a +p / -p pair of
+// rows is never cut.
+template <int ALPHA, bool SYM, typename T, int LO = 0, int HI = ALPHA>
 __device__ __forceinline__ void pass_1d(const T (&d)[ALPHA], T (&o)[ALPHA], const MatBt2& Bt)
 {
     if (SYM) {
-        // row of the point 0: even powers only
-        T s = v_mul(Bt.v[0], d[0]);
+        static_assert((LO == 0 || (LO & 1)) && (HI == ALPHA || (HI & 1)), "a pass may not cut a +p / -p pair");
+        if (LO == 0) {
+            // row of the point 0: even powers only
+            T s = v_mul(Bt.v[0], d[0]);
 #pragma unroll
-        for (int r = 2; r < ALPHA; r += 2) s = v_fma(Bt.v[r], d[r], s);
-        o[0] = s;
-        // row of the point at infinity: odd powers only
-        s = v_mul(Bt.v[(ALPHA - 1) * ALPHA + 1], d[1]);
+            for (int r = 2; r < ALPHA; r += 2) s = v_fma(Bt.v[r], d[r], s);
+            o[0] = s;
+        }
+        if (HI == ALPHA) {
+            // row of the point at infinity: odd powers only
+            T s = v_mul(Bt.v[(ALPHA - 1) * ALPHA + 1], d[1]);
 #pragma unroll
-        for (int r = 3; r < ALPHA; r += 2) s = v_fma(Bt.v[(ALPHA - 1) * ALPHA + r], d[r], s);
-        o[ALPHA - 1] = s;
+            for (int r = 3; r < ALPHA; r += 2) s = v_fma(Bt.v[(ALPHA - 1) * ALPHA + r], d[r], s);
+            o[ALPHA - 1] = s;
+        }
         // +p / -p pairs: even part E (r = 2, 4, ..), odd part O (r = 1, 3, ..); rows are E + O and E - O
 #pragma unroll
         for (int p = 1; p < ALPHA - 1; p += 2) {
+            if (p < LO || p + 1 >= HI) continue;
             T e = v_mul(Bt.v[p * ALPHA + 2], d[2]);
 #pragma unroll
             for (int r = 4; r < ALPHA - 1; r += 2) e = v_fma(Bt.v[p * ALPHA + r], d[r], e);
@@ -107,7 +115,7 @@ __device__ __forceinline__ void pass_1d(const T (&d)[ALPHA], T (&o)[ALPHA], cons
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < ALPHA; ++i) {
+        for (int i = LO; i < HI; ++i) {
             T s = v_mul(Bt.v[i * ALPHA], d[0]);
 #pragma unroll
             for (int r = 1; r < ALPHA; ++r) s = v_fma(Bt.v[i * ALPHA + r], d[r], s);
@@ -160,8 +168,9 @@ __device__ __forceinline__ void put(char* hi, char* lo, float2 v)
 
 // Row pass of one tile: h[r][j'] = sum_j d[r][j] Bt[j'][j].  p0 (and p1 for the second channel of a pair)
 // point at the 16-byte aligned vector of staged row 0 that holds the tile's first column; OFF = that
-// column's index in the vector; row_words = words between staged rows.
-template <int ALPHA, bool SYM, int OFF, typename T>
+// column's index in the vector; row_words = words between staged rows.  Only the columns LO .. HI - 1 of h are
+// computed.
+template <int ALPHA, bool SYM, int OFF, typename T, int LO = 0, int HI = ALPHA>
 __device__ __forceinline__ void rows_pass(const float* p0, const float* p1, int row_words, const MatBt2& Bt,
                                           T (&h)[ALPHA][ALPHA])
 {
@@ -184,18 +193,24 @@ __device__ __forceinline__ void rows_pass(const float* p0, const float* p1, int 
         T d[ALPHA];
 #pragma unroll
         for (int j = 0; j < ALPHA; ++j) d[j] = v_make(a[OFF + j], b[OFF + j], T());
-        pass_1d<ALPHA, SYM, T>(d, h[r], Bt);
+        pass_1d<ALPHA, SYM, T, LO, HI>(d, h[r], Bt);
+        // large tiles: keep the compiler from hoisting the loads of all rows above the arithmetic of the first,
+        // which would cost more registers than the intermediate itself
+        if (ALPHA >= 8) asm volatile("" ::: "memory");
     }
 }
 
-// Column pass and stores: V[i][j] = sum_r Bt[i][r] h[r][j], transform position xi = i * alpha + j.
-template <int ALPHA, bool SYM, int MODE, typename T>
+// Column pass and stores: V[i][j] = sum_r Bt[i][r] h[r][j], transform position xi = i * alpha + j, for the
+// columns j = LO .. HI - 1 (hi / lo point at position (0, 0)).
+template <int ALPHA, bool SYM, int MODE, typename T, int LO = 0, int HI = ALPHA>
 __device__ __forceinline__ void cols_pass_store(const T (&h)[ALPHA][ALPHA], const MatBt2& Bt, char* hi, char* lo,
                                                 long long plane_bytes)
 {
     const long long row_step = plane_bytes * ALPHA;   // from transform position (i, j) to (i + 1, j)
+    hi += plane_bytes * LO;
+    lo += plane_bytes * LO;
 #pragma unroll
-    for (int j = 0; j < ALPHA; ++j) {
+    for (int j = LO; j < HI; ++j) {
         T col[ALPHA], o[ALPHA];
 #pragma unroll
         for (int r = 0; r < ALPHA; ++r) col[r] = h[r][j];
@@ -210,6 +225,47 @@ __device__ __forceinline__ void cols_pass_store(const T (&h)[ALPHA][ALPHA], cons
         }
         hi += plane_bytes;
         lo += plane_bytes;
+    }
+}
+
+// One tile (columns LO .. HI - 1 of its transform): row pass from the staged rows, column pass, stores.
+// `off` = index of the tile's first input column in its 16-byte vector (0..3).
+template <int ALPHA, bool SYM, typename T, int LO, int HI>
+__device__ __forceinline__ void tile_columns(const float* p0, const float* p1, int row_words, int off, const MatBt2& Bt,
+                                             int mode, char* hi, char* lo, long long plane_bytes)
+{
+    T h[ALPHA][ALPHA];
+    switch (off) {
+        case 0: rows_pass<ALPHA, SYM, 0, T, LO, HI>(p0, p1, row_words, Bt, h); break;
+        case 1: rows_pass<ALPHA, SYM, 1, T, LO, HI>(p0, p1, row_words, Bt, h); break;
+        case 2: rows_pass<ALPHA, SYM, 2, T, LO, HI>(p0, p1, row_words, Bt, h); break;
+        default: rows_pass<ALPHA, SYM, 3, T, LO, HI>(p0, p1, row_words, Bt, h); break;
+    }
+    switch (mode) {
+        case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T, LO, HI>(h, Bt, hi, lo, plane_bytes); break;
+        case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T, LO, HI>(h, Bt, hi, lo, plane_bytes); break;
+        case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T, LO, HI>(h, Bt, hi, lo, plane_bytes); break;
+        case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T, LO, HI>(h, Bt, hi, lo, plane_bytes); break;
+        default: cols_pass_store<ALPHA, SYM, STORE_FP32, T, LO, HI>(h, Bt, hi, lo, plane_bytes); break;
+    }
+}
+
+// One tile.  Up to alpha = 6 the alpha x alpha intermediate stays in registers; from alpha = 8 on the tile is
+// done in two or three sweeps of at most 5 columns each (the staged rows are read once per sweep), which keeps
+// the intermediate at alpha x 5 values and the kernel clear of local-memory spills at 128 registers.
+template <int ALPHA, bool SYM, typename T>
+__device__ __forceinline__ void transform_tile(const float* p0, const float* p1, int row_words, int off, const MatBt2& Bt,
+                                               int mode, char* hi, char* lo, long long plane_bytes)
+{
+    if constexpr (ALPHA < 8) {
+        tile_columns<ALPHA, SYM, T, 0, ALPHA>(p0, p1, row_words, off, Bt, mode, hi, lo, plane_bytes);
+    } else if constexpr (ALPHA <= 10) {
+        tile_columns<ALPHA, SYM, T, 0, 5>(p0, p1, row_words, off, Bt, mode, hi, lo, plane_bytes);
+        tile_columns<ALPHA, SYM, T, 5, ALPHA>(p0, p1, row_words, off, Bt, mode, hi, lo, plane_bytes);
+    } else {
+        tile_columns<ALPHA, SYM, T, 0, 5>(p0, p1, row_words, off, Bt, mode, hi, lo, plane_bytes);
+        tile_columns<ALPHA, SYM, T, 5, 9>(p0, p1, row_words, off, Bt, mode, hi, lo, plane_bytes);
+        tile_columns<ALPHA, SYM, T, 9, ALPHA>(p0, p1, row_words, off, Bt, mode, hi, lo, plane_bytes);
     }
 }
 
@@ -367,23 +423,9 @@ input_transform_ws_kernel(const float* __restrict__ x, const __grid_constant__ C
                     const int s0 = lead + t * g.m;                         // staged column of the tile's first input column
                     const float* p0 = s_buf + (size_t)b * it.buf_words + (size_t)(PAIR ? lane : half * 32 + lane) * it.wb + (s0 & ~3);
                     const float* p1 = p0 + 32 * it.wb;
-                    T h[ALPHA][ALPHA];
-                    switch (s0 & 3) {
-                        case 0: rows_pass<ALPHA, SYM, 0, T>(p0, p1, row_words, Bt, h); break;
-                        case 1: rows_pass<ALPHA, SYM, 1, T>(p0, p1, row_words, Bt, h); break;
-                        case 2: rows_pass<ALPHA, SYM, 2, T>(p0, p1, row_words, Bt, h); break;
-                        default: rows_pass<ALPHA, SYM, 3, T>(p0, p1, row_words, Bt, h); break;
-                    }
                     const long long off = (tile * g.cin_pad + c) * eb;
-                    char* hi = V_hi + off;
-                    char* lo = V_lo ? V_lo + off : nullptr;
-                    switch (mode) {
-                        case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T>(h, Bt, hi, lo, plane_bytes); break;
-                        case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T>(h, Bt, hi, lo, plane_bytes); break;
-                        case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
-                        case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
-                        default: cols_pass_store<ALPHA, SYM, STORE_FP32, T>(h, Bt, hi, lo, plane_bytes); break;
-                    }
+                    transform_tile<ALPHA, SYM, T>(p0, p1, row_words, s0 & 3, Bt, mode, V_hi + off, V_lo ? V_lo + off : nullptr,
+                                                  plane_bytes);
                 }
             }
             __syncwarp();
@@ -496,23 +538,8 @@ input_transform_plane_kernel(const float* __restrict__ x, char* V_hi, char* V_lo
         const int s0 = pi.lead + tx * g.m - g.pad;                 // staged column of the tile's first input column
         const float* p0 = s_buf + (size_t)(PAIR ? lane : half * 32 + lane) * plane + (size_t)(ty * g.m) * pi.wp + (s0 & ~3);
         const float* p1 = p0 + (size_t)32 * plane;
-        T h[ALPHA][ALPHA];
-        switch (s0 & 3) {
-            case 0: rows_pass<ALPHA, SYM, 0, T>(p0, p1, pi.wp, Bt, h); break;
-            case 1: rows_pass<ALPHA, SYM, 1, T>(p0, p1, pi.wp, Bt, h); break;
-            case 2: rows_pass<ALPHA, SYM, 2, T>(p0, p1, pi.wp, Bt, h); break;
-            default: rows_pass<ALPHA, SYM, 3, T>(p0, p1, pi.wp, Bt, h); break;
-        }
         const long long off = (tile * g.cin_pad + c) * eb;
-        char* hi = V_hi + off;
-        char* lo = V_lo ? V_lo + off : nullptr;
-        switch (mode) {
-            case STORE_TF32: cols_pass_store<ALPHA, SYM, STORE_TF32, T>(h, Bt, hi, lo, plane_bytes); break;
-            case STORE_BF16: cols_pass_store<ALPHA, SYM, STORE_BF16, T>(h, Bt, hi, lo, plane_bytes); break;
-            case STORE_TF32_SPLIT: cols_pass_store<ALPHA, SYM, STORE_TF32_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
-            case STORE_BF16_SPLIT: cols_pass_store<ALPHA, SYM, STORE_BF16_SPLIT, T>(h, Bt, hi, lo, plane_bytes); break;
-            default: cols_pass_store<ALPHA, SYM, STORE_FP32, T>(h, Bt, hi, lo, plane_bytes); break;
-        }
+        transform_tile<ALPHA, SYM, T>(p0, p1, pi.wp, s0 & 3, Bt, mode, V_hi + off, V_lo ? V_lo + off : nullptr, plane_bytes);
     }
 }
 
