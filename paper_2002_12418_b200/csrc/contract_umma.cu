@@ -57,6 +57,10 @@ struct KernelParams {
     // a_mn mode: operand A comes from x [images][Cin][hw]; atoms of 32 pixels: full_atoms = hw / 32 whole ones
     // and a ragged one when hw % 32 != 0; tiles_per_image work items of up to four atoms cover an image
     int a_mn, hw, full_atoms, atoms_per_image, tiles_per_image;
+    // sub = MMA row tiles per work item (1; 2 in a_mn mode when an item covers up to eight atoms: both tiles use
+    // the item's U tile, which is then fetched once for 256 pixels); n_acc = accumulator buffers in tensor
+    // memory (2, or 1 when two tiles of 256 columns fill it)
+    int sub, n_acc;
 };
 
 // status codes written on a bounded wait that ran out
@@ -98,7 +102,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = kTileM * SW;                            // one V tile (128 tiles)
+    const uint32_t a_bytes = kTileM * SW * (uint32_t)p.sub;          // the item's V tile(s) (128 tiles each)
     const uint32_t b_bytes = (uint32_t)p.bn * SW;                    // one U tile (bn output channels)
     const uint32_t split = p.passes == 3 ? 2u : 1u;
     const uint32_t stage_bytes = (a_bytes + b_bytes) * split;
@@ -158,12 +162,13 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     const uint32_t sbase = smem_base + stage * stage_bytes;
                     if (p.a_mn) {
                         const int img = tb / p.tiles_per_image;
-                        const int a0 = (tb - img * p.tiles_per_image) * (kTileM / 32);       // first atom of the item
-                        const int n_full = min(kTileM / 32, max(0, p.full_atoms - a0));
-                        const bool ragged = p.full_atoms < p.atoms_per_image && a0 + kTileM / 32 >= p.atoms_per_image;
+                        const int api = (kTileM / 32) * p.sub;                               // atoms per item
+                        const int a0 = (tb - img * p.tiles_per_image) * api;                 // first atom of the item
+                        const int n_full = min(api, max(0, p.full_atoms - a0));
+                        const bool ragged = p.full_atoms < p.atoms_per_image && a0 + api >= p.atoms_per_image;
                         ptx::mbar_expect_tx(bar, (uint32_t)(n_full + (ragged ? 1 : 0)) * 4096u + b_bytes);
                         if (n_full > 0)
-                            ptx::tma_load_4d(sbase, a0 + kTileM / 32 <= p.full_atoms ? &map_v_hi : &map_v_lo, bar, 0,
+                            ptx::tma_load_4d(sbase, a0 + api <= p.full_atoms ? &map_v_hi : &map_v_lo, bar, 0,
                                              kb * k_elems, a0, img);
                         if (ragged)
                             ptx::tma_load_3d(sbase + (uint32_t)n_full * 4096u, &map_x_ragged, bar, p.full_atoms * 32,
@@ -197,7 +202,14 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     break;
                 }
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.bn;
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(p.bn * p.sub);
+                // second row tile of the item (sub = 2): only when the image has atoms left for it
+                bool second = false;
+                if (p.sub == 2) {
+                    const int tb = (int)(item % p.n_tile_blocks);
+                    const int img = tb / p.tiles_per_image;
+                    second = (tb - img * p.tiles_per_image) * 8 + 4 < p.atoms_per_image;
+                }
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full_bar[stage]), phase, abortp)) {
                         if (!*abortp) atomicCAS(p.status, 0, kErrMmaWaitFull);
@@ -214,6 +226,9 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                                                                     : desc_k<SW>(sbase + ks * 32);
                         const uint64_t b_hi = desc_k<SW>(sbase + off_b_hi + ks * 32);
                         ptx::mma_ss<KIND>(d_tmem, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
+                        if (second)
+                            ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, ptx::smem_desc_mn128_b32(sbase + 16384 + ks * 1024, 4096), b_hi,
+                                              idesc, (kb | ks) != 0 ? 1u : 0u);
                         if (split == 2) {
                             const uint64_t a_lo = desc_k<SW>(sbase + off_a_lo + ks * 32);
                             const uint64_t b_lo = desc_k<SW>(sbase + off_b_lo + ks * 32);
@@ -229,8 +244,10 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 }
                 if (!ok) break;
                 ptx::mma_commit(ptx::smem_u32(&tfull_bar[acc]));           // accumulator complete
-                acc ^= 1u;
-                if (acc == 0) acc_phase ^= 1u;
+                if (++acc == (uint32_t)p.n_acc) {
+                    acc = 0;
+                    acc_phase ^= 1u;
+                }
             }
         }
     } else {
@@ -256,9 +273,10 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 break;
             }
             ptx::tc_fence_after();
+            for (int sub = 0; sub < p.sub; ++sub) {
             const long long t = (long long)tb * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
             bool t_ok = t < p.tiles;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)p.bn;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)(p.bn * p.sub) + (uint32_t)(sub * p.bn);
             const int co0 = nb * p.bn;
             const int n_co = min(p.bn, p.Cout - co0);                        // valid output channels of this item
             // destination of channel co0 for this thread, and the distance to the next channel
@@ -269,7 +287,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 dst = p.epi.M + ((size_t)xi * p.Cout + co0) * p.epi.m_row_stride + t;
             } else if (p.a_mn) {
                 const int img = tb / p.tiles_per_image;
-                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) + q) * 32 + lane;   // this warp's atom
+                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) * p.sub + 4 * sub + q) * 32 + lane;   // this warp's atom
                 t_ok = pix < p.hw;
                 step = p.hw;
                 dst = p.epi.y + ((size_t)(t_ok ? img : 0) * p.Cout + co0) * p.hw + (t_ok ? pix : 0);
@@ -349,11 +367,14 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     dst += 16 * step;
                 }
             }
+            }   // row tiles of the item
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&tempty_bar[acc]));
-            acc ^= 1u;
-            if (acc == 0) acc_phase ^= 1u;
+            if (++acc == (uint32_t)p.n_acc) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
         }
     }
 
@@ -475,6 +496,8 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
                                 void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why)
 {
     uc->ready = false;
+    uc->sub = 1;
+    uc->n_acc = 2;
     uc->a_mn = V_hi == nullptr;        // operand A is read from x at launch time (umma_contract_setup_x)
     if (uc->a_mn && (mode != STORE_TF32 || alpha2 != 1)) {
         *why = "reading x as operand A needs single-pass TF32 and one transform position";
@@ -564,6 +587,24 @@ cudaError_t umma_contract_setup_x(UmmaContract* uc, int Cout, int Cin, int cin_p
     uc->x_cin = Cin;
     uc->x_hw = hw;
     uc->k_blocks = (Cin + 31) / 32;
+    // Images of more than four atoms: work items of up to eight atoms (two row tiles sharing one U tile) where
+    // three such stages fit and the accumulators either stay double buffered (bn <= 128) or the items make one
+    // round over the SMs (then nothing waits for the single buffer).
+    if (atoms > kTileM / 32) {
+        const int stage2 = 2 * kTileM * kSwizzleBytes + uc->bn * kSwizzleBytes;
+        int stages2 = (kSmemBudget - 1024) / stage2;
+        if (stages2 > kMaxStages) stages2 = kMaxStages;
+        const long long items2 = (long long)images * ((atoms + 7) / 8) * uc->n_co_blocks;
+        const bool dbl = 4 * uc->bn <= 512;
+        if (stages2 >= 3 && (dbl || items2 <= uc->num_sms)) {
+            uc->sub = 2;
+            uc->n_acc = dbl ? 2 : 1;
+            uc->stages = stages2;
+            int cols = 32;
+            while (cols < uc->n_acc * 2 * uc->bn) cols *= 2;
+            uc->tmem_cols = cols;
+        }
+    }
     return cudaSuccess;
 }
 
@@ -578,7 +619,10 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.hw = uc.x_hw;
     p.full_atoms = uc.x_hw / 32;
     p.atoms_per_image = (uc.x_hw + 31) / 32;
-    p.tiles_per_image = (p.atoms_per_image + kTileM / 32 - 1) / (kTileM / 32);
+    const int api = (kTileM / 32) * uc.sub;                                    // atoms per work item
+    p.tiles_per_image = (p.atoms_per_image + api - 1) / api;
+    p.sub = uc.sub;
+    p.n_acc = uc.n_acc;
     // Tensor maps over x, 128-byte swizzle with a 32-byte base.  Whole atoms: x as [image][atom][channel][32
     // pixels] (the atom stride, 128 bytes, is smaller than the channel stride), box = 32 pixels x 32 channels x
     // h atoms, h = 4 for the leading items of an image and what is left for its last item.  Ragged atom: x as
@@ -594,9 +638,9 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
     };
     CUtensorMap map_lead, map_last, map_ragged;
-    const int h_lead = p.full_atoms < kTileM / 32 ? p.full_atoms : kTileM / 32;
-    int h_last = p.full_atoms - (p.tiles_per_image - 1) * (kTileM / 32);       // whole atoms of an image's last item
-    if (h_last < 1 || h_last > kTileM / 32) h_last = h_lead;                   // (none: the map is not used)
+    const int h_lead = p.full_atoms < api ? p.full_atoms : api;
+    int h_last = p.full_atoms - (p.tiles_per_image - 1) * api;                 // whole atoms of an image's last item
+    if (h_last < 1 || h_last > api) h_last = h_lead;                           // (none: the map is not used)
     if (!encode_atoms(&map_lead, h_lead) || !encode_atoms(&map_last, h_last)) return cudaErrorInvalidValue;
     {
         const cuuint64_t dims[3] = {(cuuint64_t)uc.x_hw, (cuuint64_t)uc.x_cin, (cuuint64_t)uc.x_images};
@@ -617,7 +661,7 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.stages = uc.stages;
     p.tmem_cols = uc.tmem_cols;
     p.Cout = uc.Cout;
-    p.tiles = (long long)p.n_tile_blocks * kTileM;
+    p.tiles = (long long)p.n_tile_blocks * kTileM * uc.sub;
     p.n_items = (long long)p.n_tile_blocks * p.n_co_blocks;
     p.epi = epi;
     p.status = status;
@@ -638,6 +682,8 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     p.full_atoms = 0;
     p.atoms_per_image = 1;
     p.tiles_per_image = 1;
+    p.sub = 1;
+    p.n_acc = 2;
     p.alpha2 = uc.alpha2;
     p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
     p.n_co_blocks = uc.n_co_blocks;

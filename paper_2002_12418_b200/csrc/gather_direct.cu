@@ -693,7 +693,9 @@ __device__ __forceinline__ void dw_load_row(const float* __restrict__ p, bool ok
     }
 }
 
-template <int STRIDE, int SW, int VIN>
+// HMAX > 0 (planes of at most HMAX rows): every row of the plane is requested before the first is used, one
+// trip to memory per warp instead of one per four rows, which is what short planes (14 x 14, 7 x 7) are bound by.
+template <int STRIDE, int SW, int VIN, int HMAX = 0>
 __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __restrict__ x, const float* __restrict__ w,
                                                                const float* __restrict__ bias, float* __restrict__ y,
                                                                DirectGeom g, int strips, int bands, long long n_planes,
@@ -770,6 +772,17 @@ __global__ void __launch_bounds__(128) depthwise3x3_vec_kernel(const float* __re
     };
     float* yrow = yp + (owns ? oh0 * OWd + ocol0 : 0);                     // output row oh0 of this lane's columns
 
+    if constexpr (HMAX > 0) {
+        DwRow<VIN> rows[HMAX + 2];                    // rows[i] = input row i - 1; rows outside the plane are zero
+#pragma unroll
+        for (int i = 0; i < HMAX + 2; ++i) load(i - 1, rows[i]);
+#pragma unroll
+        for (int i = 0; i < HMAX + 2; ++i) edges(rows[i]);
+#pragma unroll
+        for (int k = 0; k < (STRIDE == 1 ? HMAX : (HMAX + 1) / 2); ++k)
+            out(yrow + k * OWd, owns && k < oh1, rows[STRIDE * k], rows[STRIDE * k + 1], rows[STRIDE * k + 2]);
+        return;
+    }
     if (STRIDE == 1) {
         DwRow<VIN> r0, r1;
         load(oh0 - 1, r0);
@@ -876,6 +889,15 @@ cudaError_t launch_direct(const float* x, const float* w, const float* bias, flo
             const long long units = groups * strips * bands;
             const long long blocks = (units + 3) / 4;
             if (units > 2147483647ll - 4) return cudaErrorInvalidValue;
+            // short planes held whole in registers: up to 16 rows with 2 columns per lane, up to 8 with 4
+            if (strips == 1 && sw == 8 && g.H <= (vin == 2 ? 16 : 8)) {
+#define MNNB_DWS_LAUNCH(ST, VI, HM) depthwise3x3_vec_kernel<ST, 8, VI, HM><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, planes, units)
+                if (vin == 4) { if (g.stride == 1) MNNB_DWS_LAUNCH(1, 4, 8); else MNNB_DWS_LAUNCH(2, 4, 8); }
+                else if (g.H <= 8) { if (g.stride == 1) MNNB_DWS_LAUNCH(1, 2, 8); else MNNB_DWS_LAUNCH(2, 2, 8); }
+                else { if (g.stride == 1) MNNB_DWS_LAUNCH(1, 2, 16); else MNNB_DWS_LAUNCH(2, 2, 16); }
+#undef MNNB_DWS_LAUNCH
+                return cudaGetLastError();
+            }
 #define MNNB_DWV_LAUNCH(ST, SWV, VI) depthwise3x3_vec_kernel<ST, SWV, VI><<<(unsigned)blocks, 128, 0, stream>>>(x, w, bias, y, g, strips, bands, planes, units)
 #define MNNB_DWV_PICK(ST, VI) do { if (sw == 8) MNNB_DWV_LAUNCH(ST, 8, VI); else if (sw == 16) MNNB_DWV_LAUNCH(ST, 16, VI); else MNNB_DWV_LAUNCH(ST, 32, VI); } while (0)
             if (g.stride == 1) {

@@ -315,7 +315,10 @@ def test_gemm_bit_exact_on_integers(torch):
 @pytest.mark.parametrize("Cin,Cout,H,W_,N", [
     (64, 128, 8, 8, 2), (24, 40, 14, 14, 3), (512, 512, 14, 14, 1), (100, 72, 6, 6, 5), (32, 16, 28, 28, 2),
     (72, 300, 9, 12, 2), (130, 260, 7, 12, 7), (8, 8, 4, 8, 1), (16, 24, 8, 16, 2), (40, 48, 10, 16, 2),
-    (33, 20, 16, 18, 1), (20, 24, 4, 9, 3)])
+    (33, 20, 16, 18, 1), (20, 24, 4, 9, 3),
+    # images of more than four atoms (work items of two row tiles): exactly eight atoms, seven and a ragged one,
+    # fifty atoms (a last item of two), two channel blocks, one buffered accumulator pair (Cout > 128)
+    (48, 64, 16, 16, 3), (16, 272, 12, 20, 2), (64, 96, 40, 40, 1), (96, 512, 14, 14, 4)])
 @pytest.mark.parametrize("lhs", [B.GEMM_LHS_PATCHES, B.GEMM_LHS_X])
 def test_gemm_left_operand_1x1(torch, Cin, Cout, H, W_, N, lhs):
     layer = W.ConvLayer("t", N, Cin, Cout, H, W_, 1, 1, 0, 1, relu=True, seed=Cin + H)
@@ -395,6 +398,25 @@ def test_generic_direct(torch, Cin, Cout, H, k, stride, pad, dil, groups):
     got, info, _ = run_layer(torch, layer, opts_for(layer, force_algo=B.ALGO_DIRECT), (x, w, b))
     assert info.algo == B.ALGO_DIRECT
     assert rel_l2(got, oracle(layer, x, w, b)) < 1e-6
+
+
+# Planes of at most 256 elements take the kernel that stages four whole planes per warp in shared memory: plane
+# counts that leave the last group partial, odd and even widths (single outputs / output pairs), both strides,
+# the smallest planes.
+@pytest.mark.parametrize("C,H,W_,N", [(13, 14, 14, 5), (9, 7, 7, 7), (6, 16, 16, 2), (5, 3, 11, 3), (3, 1, 1, 2),
+                                      (2, 2, 128, 1), (7, 15, 17, 1), (512, 14, 14, 2)])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_depthwise_small_planes(torch, C, H, W_, N, stride):
+    layer = W.ConvLayer("t", N, C, C, H, W_, 3, stride, 1, groups=C, relu=(C % 2 == 1), seed=C + H)
+    x, w, b = W.make_inputs(layer)
+    got, info, _ = run_layer(torch, layer, opts_for(layer), (x, w, b))
+    assert info.algo == B.ALGO_DIRECT
+    ref = oracle(layer, x, w, b)
+    assert got.shape == ref.shape
+    assert rel_l2(got, ref) < 1e-6
+    xi, wi, bi = W.integer_inputs(layer)
+    goti, _, _ = run_layer(torch, layer, opts_for(layer), (xi, wi, bi))
+    assert np.array_equal(goti.astype(np.float64), oracle(layer, xi, wi, bi))
 
 
 @pytest.mark.parametrize("Cout,H,Wd,relu", [(70, 30, 44, False), (32, 64, 64, True), (5, 2, 4, True), (21, 8, 12, False), (48, 100, 36, True)])
