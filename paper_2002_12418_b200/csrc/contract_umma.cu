@@ -57,10 +57,13 @@ struct KernelParams {
     // a_mn mode: operand A comes from x [images][Cin][hw]; atoms of 32 pixels: full_atoms = hw / 32 whole ones
     // and a ragged one when hw % 32 != 0; tiles_per_image work items of up to four atoms cover an image
     int a_mn, hw, full_atoms, atoms_per_image, tiles_per_image;
-    // sub = MMA row tiles per work item (1; 2 in a_mn mode when an item covers up to eight atoms: both tiles use
-    // the item's U tile, which is then fetched once for 256 pixels); n_acc = accumulator buffers in tensor
-    // memory (2, or 1 when two tiles of 256 columns fill it)
+    // sub = MMA row tiles per work item, the kernel's SUB (1; 2 in a_mn mode when an item covers up to eight
+    // atoms: both tiles use the item's U tile, which is then fetched once for 256 pixels); n_acc = accumulator
+    // buffers in tensor memory (2, or 1 when two tiles of 256 columns fill it)
     int sub, n_acc;
+    // 1: hi and lo operand tiles arrive with one copy each for V and U (maps with a hi / lo dimension, see
+    // encode_operand_pair_map); halves the copies the producer issues per stage
+    int merged;
 };
 
 // status codes written on a bounded wait that ran out
@@ -83,7 +86,7 @@ __device__ __forceinline__ uint64_t desc_k(uint32_t smem_addr)
 // SW = bytes of K per shared-memory row of an operand tile (the swizzle span): 128, or 64 where 128-byte rows
 // would leave room for two pipeline stages only (hi + lo operands with wide channel blocks): the same bytes
 // in flight in twice as many stages keep the tensor core fed across the TMA latency.
-template <int KIND, int SW>
+template <int KIND, int SW, int SUB>
 __global__ void __launch_bounds__(kThreads, 1)
 contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_constant__ CUtensorMap map_v_lo,
                      const __grid_constant__ CUtensorMap map_u_hi, const __grid_constant__ CUtensorMap map_u_lo,
@@ -102,7 +105,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = kTileM * SW * (uint32_t)p.sub;          // the item's V tile(s) (128 tiles each)
+    const uint32_t a_bytes = kTileM * SW * (uint32_t)SUB;          // the item's V tile(s) (128 tiles each)
     const uint32_t b_bytes = (uint32_t)p.bn * SW;                    // one U tile (bn output channels)
     const uint32_t split = p.passes == 3 ? 2u : 1u;
     const uint32_t stage_bytes = (a_bytes + b_bytes) * split;
@@ -162,7 +165,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     const uint32_t sbase = smem_base + stage * stage_bytes;
                     if (p.a_mn) {
                         const int img = tb / p.tiles_per_image;
-                        const int api = (kTileM / 32) * p.sub;                               // atoms per item
+                        const int api = (kTileM / 32) * SUB;                               // atoms per item
                         const int a0 = (tb - img * p.tiles_per_image) * api;                 // first atom of the item
                         const int n_full = min(api, max(0, p.full_atoms - a0));
                         const bool ragged = p.full_atoms < p.atoms_per_image && a0 + api >= p.atoms_per_image;
@@ -175,12 +178,17 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                                              kb * k_elems, img);
                     } else {
                         ptx::mbar_expect_tx(bar, stage_bytes);
-                        ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
+                        if (p.merged) ptx::tma_load_4d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM * SUB, 0, xi);
+                        else ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM * SUB, xi);
                     }
-                    ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
-                    if (split == 2) {
-                        ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM, xi);
-                        ptx::tma_load_3d(sbase + off_b_lo, &map_u_lo, bar, kb * k_elems, nb * p.bn, xi);
+                    if (p.merged) {
+                        ptx::tma_load_4d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, 0, xi);
+                    } else {
+                        ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
+                        if (split == 2) {
+                            ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM * SUB, xi);
+                            ptx::tma_load_3d(sbase + off_b_lo, &map_u_lo, bar, kb * k_elems, nb * p.bn, xi);
+                        }
                     }
                     if (++stage == (uint32_t)p.stages) {
                         stage = 0;
@@ -202,13 +210,14 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     break;
                 }
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(p.bn * p.sub);
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(p.bn * SUB);
                 // second row tile of the item (sub = 2): only when the image has atoms left for it
                 bool second = false;
-                if (p.sub == 2) {
+                if (SUB == 2) {
                     const int tb = (int)(item % p.n_tile_blocks);
                     const int img = tb / p.tiles_per_image;
-                    second = (tb - img * p.tiles_per_image) * 8 + 4 < p.atoms_per_image;
+                    second = p.a_mn ? (tb - img * p.tiles_per_image) * 8 + 4 < p.atoms_per_image
+                                    : (2ll * tb + 1) * kTileM < p.tiles;
                 }
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full_bar[stage]), phase, abortp)) {
@@ -226,14 +235,20 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                                                                     : desc_k<SW>(sbase + ks * 32);
                         const uint64_t b_hi = desc_k<SW>(sbase + off_b_hi + ks * 32);
                         ptx::mma_ss<KIND>(d_tmem, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
-                        if (second)
-                            ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, ptx::smem_desc_mn128_b32(sbase + 16384 + ks * 1024, 4096), b_hi,
-                                              idesc, (kb | ks) != 0 ? 1u : 0u);
+                        // second row tile: the next four atoms (a_mn), or the next 128 rows of the K-major tile
+                        const uint64_t a2_hi = (SW == 128 && p.a_mn) ? ptx::smem_desc_mn128_b32(sbase + 16384 + ks * 1024, 4096)
+                                                                     : desc_k<SW>(sbase + kTileM * SW + ks * 32);
+                        if (SUB == 2 && second) ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, a2_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
                         if (split == 2) {
                             const uint64_t a_lo = desc_k<SW>(sbase + off_a_lo + ks * 32);
                             const uint64_t b_lo = desc_k<SW>(sbase + off_b_lo + ks * 32);
                             ptx::mma_ss<KIND>(d_tmem, a_lo, b_hi, idesc, 1u);
                             ptx::mma_ss<KIND>(d_tmem, a_hi, b_lo, idesc, 1u);
+                            if (SUB == 2 && second) {
+                                const uint64_t a2_lo = desc_k<SW>(sbase + off_a_lo + kTileM * SW + ks * 32);
+                                ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, a2_lo, b_hi, idesc, 1u);
+                                ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, a2_hi, b_lo, idesc, 1u);
+                            }
                         }
                     }
                     ptx::mma_commit(ptx::smem_u32(&empty_bar[stage]));     // stage reusable once these MMAs retire
@@ -273,10 +288,11 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 break;
             }
             ptx::tc_fence_after();
-            for (int sub = 0; sub < p.sub; ++sub) {
-            const long long t = (long long)tb * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
+#pragma unroll
+            for (int sub = 0; sub < SUB; ++sub) {                 // row tiles of the item
+            const long long t = ((long long)tb * SUB + sub) * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
             bool t_ok = t < p.tiles;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)(p.bn * p.sub) + (uint32_t)(sub * p.bn);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)(p.bn * SUB) + (uint32_t)(sub * p.bn);
             const int co0 = nb * p.bn;
             const int n_co = min(p.bn, p.Cout - co0);                        // valid output channels of this item
             // destination of channel co0 for this thread, and the distance to the next channel
@@ -287,7 +303,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 dst = p.epi.M + ((size_t)xi * p.Cout + co0) * p.epi.m_row_stride + t;
             } else if (p.a_mn) {
                 const int img = tb / p.tiles_per_image;
-                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) * p.sub + 4 * sub + q) * 32 + lane;   // this warp's atom
+                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) * SUB + 4 * sub + q) * 32 + lane;   // this warp's atom
                 t_ok = pix < p.hw;
                 step = p.hw;
                 dst = p.epi.y + ((size_t)(t_ok ? img : 0) * p.Cout + co0) * p.hw + (t_ok ? pix : 0);
@@ -297,10 +313,11 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 dst = p.epi.y + ((size_t)img * p.Cout + co0) * p.epi.ohw + (t_ok ? t - img * p.epi.ohw : 0);
             }
             // this warp's chunks of 16 columns
-            constexpr int kParts = kEpilogueWarps / 4;
+            constexpr int col_parts = kEpilogueWarps / 4;
+            const int cpart = part;
             const int n_chunks = (n_co + 15) >> 4;
-            const int per_part = (n_chunks + kParts - 1) / kParts;
-            const int ch_begin = min(part * per_part, n_chunks), ch_end = min(ch_begin + per_part, n_chunks);
+            const int per_part = (n_chunks + col_parts - 1) / col_parts;
+            const int ch_begin = min(cpart * per_part, n_chunks), ch_end = min(ch_begin + per_part, n_chunks);
             dst += (long long)ch_begin * 16 * step;
             const bool relu = p.epi.relu != 0;
             auto store_chunk = [&](const uint32_t (&v)[16], int ch) {
@@ -453,6 +470,24 @@ static bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, 
     return r == CUDA_SUCCESS;
 }
 
+// 4-D map over a hi / lo operand pair: [planes][hi, lo][rows][k], the lo array `lo_offset_bytes` behind the hi
+// array; box = [1][2][box_rows][sw bytes of k].  One copy lands the hi tile and, right behind it, the lo tile.
+static bool encode_operand_pair_map(CUtensorMap* map, void* base_hi, long long lo_offset_bytes, int elem_bytes, long long k_len,
+                                    long long rows, long long planes, long long plane_stride_elems, int box_rows, int sw)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || lo_offset_bytes <= 0 || lo_offset_bytes % 16 != 0 || lo_offset_bytes >= (1ll << 40)) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)k_len, (cuuint64_t)rows, 2, (cuuint64_t)planes};
+    const cuuint64_t strides[3] = {(cuuint64_t)k_len * elem_bytes, (cuuint64_t)lo_offset_bytes,
+                                   (cuuint64_t)plane_stride_elems * elem_bytes};
+    const cuuint32_t box[4] = {(cuuint32_t)(sw / elem_bytes), (cuuint32_t)box_rows, 2, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    return fn(map, dt, 4, base_hi, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              sw == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 namespace wino {
 // Tensor map over x [images][C][H][W] (fp32) for the input transform's row copies, no swizzle; elements
 // outside the tensor read as zero.  Needs W * 4 to be a multiple of 16 bytes and a 16-byte aligned base.
@@ -545,7 +580,7 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     // otherwise block inside the tensor-memory allocation.
     uc->smem_bytes = kSmemBudget;
     int cols = 32;
-    while (cols < 2 * uc->bn) cols *= 2;
+    while (cols < uc->n_acc * uc->sub * uc->bn) cols *= 2;
     uc->tmem_cols = cols;
 
     const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
@@ -558,13 +593,25 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
         *why = "cuTensorMapEncodeTiled failed or is unavailable";
         return cudaErrorInvalidValue;
     }
+    // hi + lo operands that lie in one allocation each (lo behind hi): one copy per operand and stage
+    uc->merged = 0;
+    if (split == 2 && !uc->a_mn) {
+        const long long dv = static_cast<char*>(V_lo) - static_cast<char*>(V_hi), du = static_cast<char*>(U_lo) - static_cast<char*>(U_hi);
+        CUtensorMap mv, mu;
+        if (encode_operand_pair_map(&mv, V_hi, dv, eb, cin_pad, tiles_capacity, alpha2, v_plane, kTileM, sw) &&
+            encode_operand_pair_map(&mu, U_hi, du, eb, cin_pad, Cout, alpha2, u_plane, uc->bn, sw)) {
+            uc->map_v_hi = mv;
+            uc->map_u_hi = mu;
+            uc->merged = 1;
+        }
+    }
     if (uc->a_mn) uc->map_v_hi = uc->map_u_hi;      // replaced by the map over x at every launch
     if (split == 1) {
         uc->map_v_lo = uc->map_v_hi;
         uc->map_u_lo = uc->map_u_hi;
     }
-    for (auto kern : {contract_umma_kernel<0, 128>, contract_umma_kernel<1, 128>, contract_umma_kernel<0, 64>,
-                      contract_umma_kernel<1, 64>}) {
+    for (auto kern : {contract_umma_kernel<0, 128, 1>, contract_umma_kernel<1, 128, 1>, contract_umma_kernel<0, 64, 1>,
+                      contract_umma_kernel<1, 64, 1>, contract_umma_kernel<0, 128, 2>}) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         if (e != cudaSuccess) return e;
     }
@@ -588,15 +635,17 @@ cudaError_t umma_contract_setup_x(UmmaContract* uc, int Cout, int Cin, int cin_p
     uc->x_hw = hw;
     uc->k_blocks = (Cin + 31) / 32;
     // Images of more than four atoms: work items of up to eight atoms (two row tiles sharing one U tile) where
-    // three such stages fit and the accumulators either stay double buffered (bn <= 128) or the items make one
-    // round over the SMs (then nothing waits for the single buffer).
+    // three such stages fit, single-tile items would outnumber the SMs, and the accumulators either stay double
+    // buffered (bn <= 128) or the items make one round over the SMs (then nothing waits for the single buffer).
     if (atoms > kTileM / 32) {
         const int stage2 = 2 * kTileM * kSwizzleBytes + uc->bn * kSwizzleBytes;
         int stages2 = (kSmemBudget - 1024) / stage2;
         if (stages2 > kMaxStages) stages2 = kMaxStages;
+        const long long items1 = (long long)images * tiles_per_image * uc->n_co_blocks;
         const long long items2 = (long long)images * ((atoms + 7) / 8) * uc->n_co_blocks;
         const bool dbl = 4 * uc->bn <= 512;
-        if (stages2 >= 3 && (dbl || items2 <= uc->num_sms)) {
+        // (not while single-tile items leave SMs idle: small batches want the parallelism)
+        if (stages2 >= 3 && items1 > uc->num_sms && (dbl || items2 <= uc->num_sms)) {
             uc->sub = 2;
             uc->n_acc = dbl ? 2 : 1;
             uc->stages = stages2;
@@ -623,6 +672,7 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.tiles_per_image = (p.atoms_per_image + api - 1) / api;
     p.sub = uc.sub;
     p.n_acc = uc.n_acc;
+    p.merged = 0;
     // Tensor maps over x, 128-byte swizzle with a 32-byte base.  Whole atoms: x as [image][atom][channel][32
     // pixels] (the atom stride, 128 bytes, is smaller than the channel stride), box = 32 pixels x 32 channels x
     // h atoms, h = 4 for the leading items of an image and what is left for its last item.  Ragged atom: x as
@@ -666,8 +716,8 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.epi = epi;
     p.status = status;
     const long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    return launch_overlapped(contract_umma_kernel<0, 128>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
-                             map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
+    return launch_overlapped(uc.sub == 2 ? contract_umma_kernel<0, 128, 2> : contract_umma_kernel<0, 128, 1>, dim3((unsigned)grid),
+                             dim3(kThreads), (size_t)uc.smem_bytes, stream, map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
 }
 
 cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const ContractEpilogue& epi, int* status,
@@ -684,6 +734,7 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     p.tiles_per_image = 1;
     p.sub = 1;
     p.n_acc = 2;
+    p.merged = uc.merged;
     p.alpha2 = uc.alpha2;
     p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
     p.n_co_blocks = uc.n_co_blocks;
@@ -698,8 +749,8 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     p.epi = epi;
     p.status = status;
     long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    auto kern = uc.kind == 0 ? (uc.stages_sw == 64 ? contract_umma_kernel<0, 64> : contract_umma_kernel<0, 128>)
-                             : (uc.stages_sw == 64 ? contract_umma_kernel<1, 64> : contract_umma_kernel<1, 128>);
+    auto kern = uc.kind == 0 ? (uc.stages_sw == 64 ? contract_umma_kernel<0, 64, 1> : contract_umma_kernel<0, 128, 1>)
+                             : (uc.stages_sw == 64 ? contract_umma_kernel<1, 64, 1> : contract_umma_kernel<1, 128, 1>);
     return launch_overlapped(kern, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream, uc.map_v_hi,
                              uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
 }

@@ -316,9 +316,11 @@ def test_gemm_bit_exact_on_integers(torch):
     (64, 128, 8, 8, 2), (24, 40, 14, 14, 3), (512, 512, 14, 14, 1), (100, 72, 6, 6, 5), (32, 16, 28, 28, 2),
     (72, 300, 9, 12, 2), (130, 260, 7, 12, 7), (8, 8, 4, 8, 1), (16, 24, 8, 16, 2), (40, 48, 10, 16, 2),
     (33, 20, 16, 18, 1), (20, 24, 4, 9, 3),
-    # images of more than four atoms (work items of two row tiles): exactly eight atoms, seven and a ragged one,
-    # fifty atoms (a last item of two), two channel blocks, one buffered accumulator pair (Cout > 128)
-    (48, 64, 16, 16, 3), (16, 272, 12, 20, 2), (64, 96, 40, 40, 1), (96, 512, 14, 14, 4)])
+    # images of more than four atoms: exactly eight atoms, seven and a ragged one, fifty atoms, two channel blocks
+    (48, 64, 16, 16, 3), (16, 272, 12, 20, 2), (64, 96, 40, 40, 1), (96, 512, 14, 14, 4),
+    # enough single-tile items to fill the machine, which is when the two-tile items are chosen: double-buffered
+    # accumulators (Cout <= 128), one buffer (Cout 512), five atoms, twenty-five atoms
+    (32, 64, 14, 14, 80), (32, 512, 14, 14, 40), (16, 32, 10, 16, 80), (16, 16, 28, 28, 24)])
 @pytest.mark.parametrize("lhs", [B.GEMM_LHS_PATCHES, B.GEMM_LHS_X])
 def test_gemm_left_operand_1x1(torch, Cin, Cout, H, W_, N, lhs):
     layer = W.ConvLayer("t", N, Cin, Cout, H, W_, 1, 1, 0, 1, relu=True, seed=Cin + H)
