@@ -57,10 +57,6 @@ struct KernelParams {
     // a_mn mode: operand A comes from x [images][Cin][hw]; atoms of 32 pixels: full_atoms = hw / 32 whole ones
     // and a ragged one when hw % 32 != 0; tiles_per_image work items of up to four atoms cover an image
     int a_mn, hw, full_atoms, atoms_per_image, tiles_per_image;
-    // sub = MMA row tiles per work item, the kernel's SUB (1; 2 in a_mn mode when an item covers up to eight
-    // atoms: both tiles use the item's U tile, which is then fetched once for 256 pixels); n_acc = accumulator
-    // buffers in tensor memory (2, or 1 when two tiles of 256 columns fill it)
-    int sub, n_acc;
     // 1: hi and lo operand tiles arrive with one copy each for V and U (maps with a hi / lo dimension, see
     // encode_operand_pair_map); halves the copies the producer issues per stage
     int merged;
@@ -86,7 +82,7 @@ __device__ __forceinline__ uint64_t desc_k(uint32_t smem_addr)
 // SW = bytes of K per shared-memory row of an operand tile (the swizzle span): 128, or 64 where 128-byte rows
 // would leave room for two pipeline stages only (hi + lo operands with wide channel blocks): the same bytes
 // in flight in twice as many stages keep the tensor core fed across the TMA latency.
-template <int KIND, int SW, int SUB>
+template <int KIND, int SW>
 __global__ void __launch_bounds__(kThreads, 1)
 contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_constant__ CUtensorMap map_v_lo,
                      const __grid_constant__ CUtensorMap map_u_hi, const __grid_constant__ CUtensorMap map_u_lo,
@@ -105,7 +101,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = kTileM * SW * (uint32_t)SUB;          // the item's V tile(s) (128 tiles each)
+    const uint32_t a_bytes = kTileM * SW;                            // one V tile (128 tiles)
     const uint32_t b_bytes = (uint32_t)p.bn * SW;                    // one U tile (bn output channels)
     const uint32_t split = p.passes == 3 ? 2u : 1u;
     const uint32_t stage_bytes = (a_bytes + b_bytes) * split;
@@ -165,28 +161,27 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     const uint32_t sbase = smem_base + stage * stage_bytes;
                     if (p.a_mn) {
                         const int img = tb / p.tiles_per_image;
-                        const int api = (kTileM / 32) * SUB;                               // atoms per item
-                        const int a0 = (tb - img * p.tiles_per_image) * api;                 // first atom of the item
-                        const int n_full = min(api, max(0, p.full_atoms - a0));
-                        const bool ragged = p.full_atoms < p.atoms_per_image && a0 + api >= p.atoms_per_image;
+                        const int a0 = (tb - img * p.tiles_per_image) * (kTileM / 32);       // first atom of the item
+                        const int n_full = min(kTileM / 32, max(0, p.full_atoms - a0));
+                        const bool ragged = p.full_atoms < p.atoms_per_image && a0 + kTileM / 32 >= p.atoms_per_image;
                         ptx::mbar_expect_tx(bar, (uint32_t)(n_full + (ragged ? 1 : 0)) * 4096u + b_bytes);
                         if (n_full > 0)
-                            ptx::tma_load_4d(sbase, a0 + api <= p.full_atoms ? &map_v_hi : &map_v_lo, bar, 0,
+                            ptx::tma_load_4d(sbase, a0 + kTileM / 32 <= p.full_atoms ? &map_v_hi : &map_v_lo, bar, 0,
                                              kb * k_elems, a0, img);
                         if (ragged)
                             ptx::tma_load_3d(sbase + (uint32_t)n_full * 4096u, &map_x_ragged, bar, p.full_atoms * 32,
                                              kb * k_elems, img);
                     } else {
                         ptx::mbar_expect_tx(bar, stage_bytes);
-                        if (p.merged) ptx::tma_load_4d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM * SUB, 0, xi);
-                        else ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM * SUB, xi);
+                        if (p.merged) ptx::tma_load_4d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, 0, xi);
+                        else ptx::tma_load_3d(sbase, &map_v_hi, bar, kb * k_elems, tb * kTileM, xi);
                     }
                     if (p.merged) {
                         ptx::tma_load_4d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, 0, xi);
                     } else {
                         ptx::tma_load_3d(sbase + off_b_hi, &map_u_hi, bar, kb * k_elems, nb * p.bn, xi);
                         if (split == 2) {
-                            ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM * SUB, xi);
+                            ptx::tma_load_3d(sbase + off_a_lo, &map_v_lo, bar, kb * k_elems, tb * kTileM, xi);
                             ptx::tma_load_3d(sbase + off_b_lo, &map_u_lo, bar, kb * k_elems, nb * p.bn, xi);
                         }
                     }
@@ -210,15 +205,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     break;
                 }
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(p.bn * SUB);
-                // second row tile of the item (sub = 2): only when the image has atoms left for it
-                bool second = false;
-                if (SUB == 2) {
-                    const int tb = (int)(item % p.n_tile_blocks);
-                    const int img = tb / p.tiles_per_image;
-                    second = p.a_mn ? (tb - img * p.tiles_per_image) * 8 + 4 < p.atoms_per_image
-                                    : (2ll * tb + 1) * kTileM < p.tiles;
-                }
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.bn;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full_bar[stage]), phase, abortp)) {
                         if (!*abortp) atomicCAS(p.status, 0, kErrMmaWaitFull);
@@ -235,20 +222,11 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                                                                     : desc_k<SW>(sbase + ks * 32);
                         const uint64_t b_hi = desc_k<SW>(sbase + off_b_hi + ks * 32);
                         ptx::mma_ss<KIND>(d_tmem, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
-                        // second row tile: the next four atoms (a_mn), or the next 128 rows of the K-major tile
-                        const uint64_t a2_hi = (SW == 128 && p.a_mn) ? ptx::smem_desc_mn128_b32(sbase + 16384 + ks * 1024, 4096)
-                                                                     : desc_k<SW>(sbase + kTileM * SW + ks * 32);
-                        if (SUB == 2 && second) ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, a2_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
                         if (split == 2) {
                             const uint64_t a_lo = desc_k<SW>(sbase + off_a_lo + ks * 32);
                             const uint64_t b_lo = desc_k<SW>(sbase + off_b_lo + ks * 32);
                             ptx::mma_ss<KIND>(d_tmem, a_lo, b_hi, idesc, 1u);
                             ptx::mma_ss<KIND>(d_tmem, a_hi, b_lo, idesc, 1u);
-                            if (SUB == 2 && second) {
-                                const uint64_t a2_lo = desc_k<SW>(sbase + off_a_lo + kTileM * SW + ks * 32);
-                                ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, a2_lo, b_hi, idesc, 1u);
-                                ptx::mma_ss<KIND>(d_tmem + (uint32_t)p.bn, a2_hi, b_lo, idesc, 1u);
-                            }
                         }
                     }
                     ptx::mma_commit(ptx::smem_u32(&empty_bar[stage]));     // stage reusable once these MMAs retire
@@ -259,10 +237,8 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 }
                 if (!ok) break;
                 ptx::mma_commit(ptx::smem_u32(&tfull_bar[acc]));           // accumulator complete
-                if (++acc == (uint32_t)p.n_acc) {
-                    acc = 0;
-                    acc_phase ^= 1u;
-                }
+                acc ^= 1u;
+                if (acc == 0) acc_phase ^= 1u;
             }
         }
     } else {
@@ -288,11 +264,9 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 break;
             }
             ptx::tc_fence_after();
-#pragma unroll
-            for (int sub = 0; sub < SUB; ++sub) {                 // row tiles of the item
-            const long long t = ((long long)tb * SUB + sub) * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
+            const long long t = (long long)tb * kTileM + q * 32 + lane;      // this thread's tile (or GEMM column)
             bool t_ok = t < p.tiles;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)(p.bn * SUB) + (uint32_t)(sub * p.bn);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)p.bn;
             const int co0 = nb * p.bn;
             const int n_co = min(p.bn, p.Cout - co0);                        // valid output channels of this item
             // destination of channel co0 for this thread, and the distance to the next channel
@@ -303,7 +277,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 dst = p.epi.M + ((size_t)xi * p.Cout + co0) * p.epi.m_row_stride + t;
             } else if (p.a_mn) {
                 const int img = tb / p.tiles_per_image;
-                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) * SUB + 4 * sub + q) * 32 + lane;   // this warp's atom
+                const int pix = ((tb - img * p.tiles_per_image) * (kTileM / 32) + q) * 32 + lane;   // this warp's atom
                 t_ok = pix < p.hw;
                 step = p.hw;
                 dst = p.epi.y + ((size_t)(t_ok ? img : 0) * p.Cout + co0) * p.hw + (t_ok ? pix : 0);
@@ -313,11 +287,10 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 dst = p.epi.y + ((size_t)img * p.Cout + co0) * p.epi.ohw + (t_ok ? t - img * p.epi.ohw : 0);
             }
             // this warp's chunks of 16 columns
-            constexpr int col_parts = kEpilogueWarps / 4;
-            const int cpart = part;
+            constexpr int kParts = kEpilogueWarps / 4;
             const int n_chunks = (n_co + 15) >> 4;
-            const int per_part = (n_chunks + col_parts - 1) / col_parts;
-            const int ch_begin = min(cpart * per_part, n_chunks), ch_end = min(ch_begin + per_part, n_chunks);
+            const int per_part = (n_chunks + kParts - 1) / kParts;
+            const int ch_begin = min(part * per_part, n_chunks), ch_end = min(ch_begin + per_part, n_chunks);
             dst += (long long)ch_begin * 16 * step;
             const bool relu = p.epi.relu != 0;
             auto store_chunk = [&](const uint32_t (&v)[16], int ch) {
@@ -384,14 +357,11 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     dst += 16 * step;
                 }
             }
-            }   // row tiles of the item
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&tempty_bar[acc]));
-            if (++acc == (uint32_t)p.n_acc) {
-                acc = 0;
-                acc_phase ^= 1u;
-            }
+            acc ^= 1u;
+            if (acc == 0) acc_phase ^= 1u;
         }
     }
 
@@ -531,8 +501,6 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
                                 void* U_hi, void* U_lo, void* V_hi, void* V_lo, const char** why)
 {
     uc->ready = false;
-    uc->sub = 1;
-    uc->n_acc = 2;
     uc->a_mn = V_hi == nullptr;        // operand A is read from x at launch time (umma_contract_setup_x)
     if (uc->a_mn && (mode != STORE_TF32 || alpha2 != 1)) {
         *why = "reading x as operand A needs single-pass TF32 and one transform position";
@@ -580,7 +548,7 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
     // otherwise block inside the tensor-memory allocation.
     uc->smem_bytes = kSmemBudget;
     int cols = 32;
-    while (cols < uc->n_acc * uc->sub * uc->bn) cols *= 2;
+    while (cols < 2 * uc->bn) cols *= 2;
     uc->tmem_cols = cols;
 
     const long long u_plane = (long long)Cout * cin_pad, v_plane = tiles_capacity * cin_pad;
@@ -610,8 +578,8 @@ cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout
         uc->map_v_lo = uc->map_v_hi;
         uc->map_u_lo = uc->map_u_hi;
     }
-    for (auto kern : {contract_umma_kernel<0, 128, 1>, contract_umma_kernel<1, 128, 1>, contract_umma_kernel<0, 64, 1>,
-                      contract_umma_kernel<1, 64, 1>, contract_umma_kernel<0, 128, 2>}) {
+    for (auto kern : {contract_umma_kernel<0, 128>, contract_umma_kernel<1, 128>, contract_umma_kernel<0, 64>,
+                      contract_umma_kernel<1, 64>}) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         if (e != cudaSuccess) return e;
     }
@@ -634,26 +602,6 @@ cudaError_t umma_contract_setup_x(UmmaContract* uc, int Cout, int Cin, int cin_p
     uc->x_cin = Cin;
     uc->x_hw = hw;
     uc->k_blocks = (Cin + 31) / 32;
-    // Images of more than four atoms: work items of up to eight atoms (two row tiles sharing one U tile) where
-    // three such stages fit, single-tile items would outnumber the SMs, and the accumulators either stay double
-    // buffered (bn <= 128) or the items make one round over the SMs (then nothing waits for the single buffer).
-    if (atoms > kTileM / 32) {
-        const int stage2 = 2 * kTileM * kSwizzleBytes + uc->bn * kSwizzleBytes;
-        int stages2 = (kSmemBudget - 1024) / stage2;
-        if (stages2 > kMaxStages) stages2 = kMaxStages;
-        const long long items1 = (long long)images * tiles_per_image * uc->n_co_blocks;
-        const long long items2 = (long long)images * ((atoms + 7) / 8) * uc->n_co_blocks;
-        const bool dbl = 4 * uc->bn <= 512;
-        // (not while single-tile items leave SMs idle: small batches want the parallelism)
-        if (stages2 >= 3 && items1 > uc->num_sms && (dbl || items2 <= uc->num_sms)) {
-            uc->sub = 2;
-            uc->n_acc = dbl ? 2 : 1;
-            uc->stages = stages2;
-            int cols = 32;
-            while (cols < uc->n_acc * 2 * uc->bn) cols *= 2;
-            uc->tmem_cols = cols;
-        }
-    }
     return cudaSuccess;
 }
 
@@ -665,14 +613,11 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     if (!fn) return cudaErrorInvalidValue;
     KernelParams p;
     p.a_mn = 1;
+    p.merged = 0;
     p.hw = uc.x_hw;
     p.full_atoms = uc.x_hw / 32;
     p.atoms_per_image = (uc.x_hw + 31) / 32;
-    const int api = (kTileM / 32) * uc.sub;                                    // atoms per work item
-    p.tiles_per_image = (p.atoms_per_image + api - 1) / api;
-    p.sub = uc.sub;
-    p.n_acc = uc.n_acc;
-    p.merged = 0;
+    p.tiles_per_image = (p.atoms_per_image + kTileM / 32 - 1) / (kTileM / 32);
     // Tensor maps over x, 128-byte swizzle with a 32-byte base.  Whole atoms: x as [image][atom][channel][32
     // pixels] (the atom stride, 128 bytes, is smaller than the channel stride), box = 32 pixels x 32 channels x
     // h atoms, h = 4 for the leading items of an image and what is left for its last item.  Ragged atom: x as
@@ -688,9 +633,9 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
     };
     CUtensorMap map_lead, map_last, map_ragged;
-    const int h_lead = p.full_atoms < api ? p.full_atoms : api;
-    int h_last = p.full_atoms - (p.tiles_per_image - 1) * api;                 // whole atoms of an image's last item
-    if (h_last < 1 || h_last > api) h_last = h_lead;                           // (none: the map is not used)
+    const int h_lead = p.full_atoms < kTileM / 32 ? p.full_atoms : kTileM / 32;
+    int h_last = p.full_atoms - (p.tiles_per_image - 1) * (kTileM / 32);       // whole atoms of an image's last item
+    if (h_last < 1 || h_last > kTileM / 32) h_last = h_lead;                   // (none: the map is not used)
     if (!encode_atoms(&map_lead, h_lead) || !encode_atoms(&map_last, h_last)) return cudaErrorInvalidValue;
     {
         const cuuint64_t dims[3] = {(cuuint64_t)uc.x_hw, (cuuint64_t)uc.x_cin, (cuuint64_t)uc.x_images};
@@ -711,13 +656,13 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.stages = uc.stages;
     p.tmem_cols = uc.tmem_cols;
     p.Cout = uc.Cout;
-    p.tiles = (long long)p.n_tile_blocks * kTileM * uc.sub;
+    p.tiles = (long long)p.n_tile_blocks * kTileM;
     p.n_items = (long long)p.n_tile_blocks * p.n_co_blocks;
     p.epi = epi;
     p.status = status;
     const long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    return launch_overlapped(uc.sub == 2 ? contract_umma_kernel<0, 128, 2> : contract_umma_kernel<0, 128, 1>, dim3((unsigned)grid),
-                             dim3(kThreads), (size_t)uc.smem_bytes, stream, map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
+    return launch_overlapped(contract_umma_kernel<0, 128>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
+                             map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
 }
 
 cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const ContractEpilogue& epi, int* status,
@@ -728,13 +673,11 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     if (tiles > uc.tiles_capacity) return cudaErrorInvalidValue;
     KernelParams p;
     p.a_mn = 0;
+    p.merged = uc.merged;
     p.hw = 0;
     p.full_atoms = 0;
     p.atoms_per_image = 1;
     p.tiles_per_image = 1;
-    p.sub = 1;
-    p.n_acc = 2;
-    p.merged = uc.merged;
     p.alpha2 = uc.alpha2;
     p.n_tile_blocks = (int)((tiles + kTileM - 1) / kTileM);
     p.n_co_blocks = uc.n_co_blocks;
@@ -749,8 +692,8 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     p.epi = epi;
     p.status = status;
     long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    auto kern = uc.kind == 0 ? (uc.stages_sw == 64 ? contract_umma_kernel<0, 64, 1> : contract_umma_kernel<0, 128, 1>)
-                             : (uc.stages_sw == 64 ? contract_umma_kernel<1, 64, 1> : contract_umma_kernel<1, 128, 1>);
+    auto kern = uc.kind == 0 ? (uc.stages_sw == 64 ? contract_umma_kernel<0, 64> : contract_umma_kernel<0, 128>)
+                             : (uc.stages_sw == 64 ? contract_umma_kernel<1, 64> : contract_umma_kernel<1, 128>);
     return launch_overlapped(kern, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream, uc.map_v_hi,
                              uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
 }

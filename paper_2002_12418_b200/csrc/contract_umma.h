@@ -25,7 +25,6 @@ struct UmmaContract {
     bool a_mn = false;                 // operand A is x itself (1x1 stride-1 convolution), see umma_contract_setup_x
     int x_images = 0, x_cin = 0, x_hw = 0;
     int merged = 0;                    // hi and lo tiles of an operand arrive with one copy (maps with a hi / lo dimension)
-    int sub = 1, n_acc = 2;            // row tiles per work item and accumulator buffers (umma_contract_setup_x)
     bool ready = false;
 };
 // Encodes the tensor maps for U/V at the given device addresses.  Returns a CUDA error or cudaSuccess;

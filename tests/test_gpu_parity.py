@@ -318,8 +318,8 @@ def test_gemm_bit_exact_on_integers(torch):
     (33, 20, 16, 18, 1), (20, 24, 4, 9, 3),
     # images of more than four atoms: exactly eight atoms, seven and a ragged one, fifty atoms, two channel blocks
     (48, 64, 16, 16, 3), (16, 272, 12, 20, 2), (64, 96, 40, 40, 1), (96, 512, 14, 14, 4),
-    # enough single-tile items to fill the machine, which is when the two-tile items are chosen: double-buffered
-    # accumulators (Cout <= 128), one buffer (Cout 512), five atoms, twenty-five atoms
+    # more work items than SMs (several items per CTA, both accumulator buffers in use): Cout 64 and 512, five
+    # atoms, twenty-five atoms
     (32, 64, 14, 14, 80), (32, 512, 14, 14, 40), (16, 32, 10, 16, 80), (16, 16, 28, 28, 24)])
 @pytest.mark.parametrize("lhs", [B.GEMM_LHS_PATCHES, B.GEMM_LHS_X])
 def test_gemm_left_operand_1x1(torch, Cin, Cout, H, W_, N, lhs):
