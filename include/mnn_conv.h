@@ -287,6 +287,8 @@ MNN_API int mnn_strassen_rule(long long m, long long n, long long k);
  * consts[6] L2 bytes usable for one chunk     consts[7] number of SMs
  * consts[8] attoseconds per flop of the direct kernel
  * consts[9] attoseconds per flop of the direct kernel for layers with at most 4 input channels
+ *            (measured on 3 -> 32, 3x3, stride 2, padding 1, which has a kernel of its own; the other shapes
+ *            with at most 4 input channels are booked at twice this figure)
  *           (0 = use consts[8])
  * consts[10] attoseconds per byte of transformed weights delivered from L2 to ONE SM (fused Winograd kernel)
  * consts[11] picoseconds the fused kernel's tensor work takes per block of 32 input channels of one work item

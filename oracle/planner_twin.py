@@ -130,7 +130,12 @@ def direct_cost(L: Layer, c) -> int:
     # when its transposed weights fit 160 KiB of shared memory
     few_channels = (L.groups == 1 and L.Cin <= 4 and c[9] > 0 and L.N <= 65535
                     and L.Cin * L.k * L.k * (cdiv(L.Cout, 32) * 32) * 4 <= 160 * 1024)
-    return kernel_ps(c, mem_as=traffic * c[0], alu_as=flops * (c[9] if few_channels else c[8]))
+    # c[9] is the rate of the 3 -> Cout, 3x3, stride 2, padding 1 layer on even H and W a multiple of 4 (weights
+    # within 48 KiB), which has its own kernel; the other few-channel shapes run at half that rate
+    fast = (L.Cin == 3 and L.k == 3 and L.stride == 2 and L.pad == 1 and L.dil == 1 and L.H % 2 == 0 and L.W % 4 == 0
+            and 27 * (cdiv(L.Cout, 32) * 32) * 4 <= 48 * 1024)
+    rate = (c[9] if fast else 2 * c[9]) if few_channels else c[8]
+    return kernel_ps(c, mem_as=traffic * c[0], alu_as=flops * rate)
 
 
 # ---------------------------------------------------------------------------------------

@@ -52,7 +52,7 @@ Calibration default_calibration()
     c.c[6] = 80ll << 20;  // L2 bytes one chunk's V + M may occupy
     c.c[7] = 148;         // SMs
     c.c[8] = 571000;      // as per flop of the direct kernel (~3.5 TFLOP/s)
-    c.c[9] = 60000;       // as per flop of the direct kernel for Cin <= 4 (~17 TFLOP/s)
+    c.c[9] = 31000;       // as per flop of the 3 -> Cout 3x3 stride-2 kernel (~32 TFLOP/s); other Cin <= 4 shapes: twice that
     c.c[10] = 23000000;   // as per byte of U delivered to one SM by the fused kernel's weight stream (~43 GB/s per SM)
     c.c[11] = 6000000;    // ps per 32-channel block of a fused work item (64 MMAs of 128 x 32 x 8 at ~90 ns each)
     c.c[12] = 4300000;    // ps of epilogue per fused work item
@@ -309,7 +309,11 @@ uint64_t direct_cost(const LayerShape& s, const Calibration& cal)
     // layers with at most 4 input channels (groups 1) run a dedicated kernel with its own rate (consts[9])
     const bool stem = s.groups == 1 && s.Cin <= 4 && cal.c[9] > 0 &&
                       (long long)s.Cin * s.k * s.k * ((s.Cout + 31) / 32 * 32) * 4 <= 160 * 1024 && s.N <= 65535;
-    const uint64_t rate = (uint64_t)(stem ? cal.c[9] : cal.c[8]);
+    // consts[9] is measured on the 3 -> 32, 3x3, stride 2 layer, which has a kernel of its own (blocks of output
+    // pixels per thread); the other few-channel shapes run the one-pixel kernel at half that rate
+    const bool pixel_blocks = s.Cin == 3 && s.k == 3 && s.stride == 2 && s.pad == 1 && s.dil == 1 && s.H % 2 == 0 &&
+                              s.W % 4 == 0 && (long long)27 * ((s.Cout + 31) / 32 * 32) * 4 <= 48 * 1024;
+    const uint64_t rate = (uint64_t)(stem ? (pixel_blocks ? cal.c[9] : 2 * cal.c[9]) : cal.c[8]);
     return kernel_ps((u128)(x_bytes + y_bytes + w_bytes) * (uint64_t)cal.c[0], 0, (u128)flops * rate, cal);
 }
 

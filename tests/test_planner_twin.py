@@ -219,8 +219,15 @@ def test_direct_cost_by_hand():
     L = T.Layer(1, 2, 3, 4, 4, 3, 1, 1)
     traffic = 4 * (2 * 16 + 3 * 16 + 3 * 2 * 9)            # 536 bytes
     flops = 2 * 3 * 2 * 16 * 9                              # 1728
-    # two input channels: the few-channel rate c[9]
-    assert T.direct_cost(L, CAL) == max(traffic * 100000, flops * 50000) // 10 ** 6 + 3000000
+    # two input channels: twice the few-channel rate constant c[9] (c[9] itself is the 3 -> Cout 3x3 stride-2 kernel's)
+    assert T.direct_cost(L, CAL) == max(traffic * 100000, flops * 2 * 50000) // 10 ** 6 + 3000000
+    Ls = T.Layer(2, 3, 32, 8, 8, 3, 2, 1)                   # that kernel's shape: 4 x 4 outputs
+    tr = 4 * (2 * 3 * 64 + 2 * 32 * 16 + 32 * 27)
+    fl = 2 * 2 * 32 * 3 * 16 * 9
+    assert T.direct_cost(Ls, CAL) == max(tr * 100000, fl * 50000) // 10 ** 6 + 3000000
+    assert T.direct_cost(T.Layer(2, 3, 32, 8, 8, 3, 1, 1), CAL) > 0 and \
+        T.direct_cost(T.Layer(2, 3, 32, 8, 6, 3, 2, 1), CAL) == \
+        max(4 * (2 * 3 * 48 + 2 * 32 * 12 + 32 * 27) * 100000, 2 * 2 * 32 * 3 * 12 * 9 * 2 * 50000) // 10 ** 6 + 3000000
     L8 = T.Layer(1, 8, 3, 4, 4, 3, 1, 1)
     assert T.direct_cost(L8, CAL) == max(4 * (8 * 16 + 48 + 3 * 8 * 9) * 100000, 2 * 3 * 8 * 16 * 9 * 500000) // 10 ** 6 + 3000000
 
