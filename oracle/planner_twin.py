@@ -238,11 +238,18 @@ def winograd_cost(L: Layer, m: int, operand: int, passes: int, c):
     c_vm = c[1] if fits_l2 >= chunk else c[0]
     # ALU work of the transforms: 2 alpha^3 multiply-adds per (tile, channel) on the input side (the first term
     # of Eq. 2), m alpha (alpha + m) on the output side (its third term); from alpha = 8 a lane holds one channel
-    # instead of a pair (x2), from alpha = 10 the tile no longer fits the register file (x4; x8 at alpha = 12)
-    crowding = 8 if alpha >= 12 else (4 if alpha >= 10 else (2 if alpha >= 8 else 1))
-    t_in = kernel_ps(c, mem_as=x * c[0] + v * c_vm, alu_as=crowding * 4 * alpha * a2 * n * tiles_img * L.Cin * c[4])
-    t_con = kernel_ps(c, mem_as=(v + mm) * c_vm + u * c[0],
-                      tensor_as=2 * a2 * L.Cout * Cp * n * tiles_img * passes * _tensor_rate(c, operand))
+    # instead of a pair and sweeps over the tile's columns: x2 at alpha = 8, x2.25 at alpha = 10, x4 at alpha = 12
+    # (in quarters: 8, 9, 16 against 4)
+    quarters = 16 if alpha >= 12 else (9 if alpha >= 10 else (8 if alpha >= 8 else 4))
+    t_in = kernel_ps(c, mem_as=x * c[0] + v * c_vm, alu_as=quarters * alpha * a2 * n * tiles_img * L.Cin * c[4])
+    # the contraction's work items (128 tiles x bn channels x one position) go over the SMs in rounds, and the
+    # tensor time is that of full rounds
+    sms = c[7] if c[7] > 0 else 148
+    tile_blocks = cdiv(n * tiles_img, 128)
+    _, co_blocks = contraction_tiling(tile_blocks, a2, L.Cout, sms)
+    items = tile_blocks * co_blocks * a2
+    tensor = 2 * a2 * L.Cout * Cp * n * tiles_img * passes * _tensor_rate(c, operand) // items * (cdiv(items, sms) * sms)
+    t_con = kernel_ps(c, mem_as=(v + mm) * c_vm + u * c[0], tensor_as=tensor)
     t_out = kernel_ps(c, mem_as=mm * c_vm + y * c[0], alu_as=2 * m * alpha * (alpha + m) * n * tiles_img * L.Cout * c[4])
     return chunk, n_chunks, sat(n_chunks * sat(t_in + t_con + t_out))
 

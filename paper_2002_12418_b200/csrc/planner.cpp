@@ -416,13 +416,21 @@ uint64_t winograd_chunk_cost(const LayerShape& s, int m, int operand, int passes
     const uint64_t cV = (uint64_t)(resident ? cal.c[1] : cal.c[0]);
     const uint64_t c0 = (uint64_t)cal.c[0], cA = (uint64_t)cal.c[4];
     // from alpha = 8 on a lane of the input transform holds one channel instead of a packed pair (twice the ALU
-    // time); from alpha = 10 on the tile no longer fits the register file (measured about twice that again, and
-    // twice again at alpha = 12)
+    // time) and does the tile in sweeps of columns; measured against the pair form: x 2 at alpha = 8, x 2.25 at
+    // alpha = 10, x 4 at alpha = 12 (quarters: 8, 9, 16)
     const u128 tile_channels_in = (u128)n * tiles_img * (uint64_t)s.Cin, tile_channels_out = (u128)n * tiles_img * (uint64_t)s.Cout;
-    const u128 in_alu = (alpha >= 12 ? 8u : (alpha >= 10 ? 4u : (alpha >= 8 ? 2u : 1u))) * 4u * alpha * a2 * tile_channels_in * cA;
+    const u128 in_alu = (alpha >= 12 ? 16u : (alpha >= 10 ? 9u : (alpha >= 8 ? 8u : 4u))) * alpha * a2 * tile_channels_in * cA;
     const uint64_t in = kernel_ps((u128)x_bytes * c0 + (u128)v_bytes * cV, 0, in_alu, cal);
-    const uint64_t con = kernel_ps((u128)(v_bytes + m_bytes) * cV + (u128)u_bytes * c0,
-                                   2u * a2 * Cp * tile_channels_out * (uint64_t)passes * tensor_as(operand, cal), 0, cal);
+    // the contraction's work items (128 tiles x bn channels x one position) run in rounds over the SMs: its
+    // tensor time is that of full rounds
+    const uint64_t sms = cal.c[7] > 0 ? (uint64_t)cal.c[7] : 148;
+    const uint64_t tile_blocks = ceil_div(n * tiles_img, 128);
+    int bn = 0, co_blocks = 1;
+    contract_tiling((long long)tile_blocks, (int)a2, s.Cout, (int)sms, &bn, &co_blocks);
+    const uint64_t items = tile_blocks * (uint64_t)co_blocks * a2, rounds = ceil_div(items, sms);
+    // (per item first: the product with rounds x SMs then stays below twice the plain tensor time)
+    const u128 con_tensor = 2u * a2 * Cp * tile_channels_out * (uint64_t)passes * tensor_as(operand, cal) / items * (rounds * sms);
+    const uint64_t con = kernel_ps((u128)(v_bytes + m_bytes) * cV + (u128)u_bytes * c0, con_tensor, 0, cal);
     const uint64_t out = kernel_ps((u128)m_bytes * cV + (u128)y_bytes * c0, 0,
                                    2u * (uint64_t)m * alpha * (alpha + m) * tile_channels_out * cA, cal);
     return saturate((u128)in + con + out);

@@ -248,6 +248,34 @@ def test_winograd_cost_by_hand():
     assert cost == t_in + t_con + t_out
 
 
+def test_winograd_rounds_and_large_tiles_by_hand():
+    """The contraction's tensor time counts full rounds of work items over the SMs, and the input transform's
+    ALU term grows with alpha in the measured steps (quarters 4, 8, 9, 16).  Constants chosen so that the
+    tensor and ALU terms decide: memory free, 1e9 as per tensor flop, 1e9 as per ALU flop, 7 SMs."""
+    cal = [0, 0, 10 ** 9, 10 ** 9, 10 ** 9, 1000, 1 << 40, 7, 1, 1, 0, 0, 0, 0, 0, 0]
+    # 1 image, 8 -> 16 channels, 4 x 4 outputs, m = 2: alpha 4, 4 tiles: 1 tile block x 1 channel block x 16
+    # positions = 16 items on 7 SMs = 3 rounds
+    L = T.Layer(1, 8, 16, 4, 4, 3, 1, 1)
+    _, _, cost = T.winograd_cost(L, 2, T.OPERAND_TF32, 1, cal)
+    flops_con = 2 * 16 * 16 * 8 * 4
+    t_con = (flops_con * 10 ** 9 // 16 * 21) // 10 ** 6 + 1000
+    t_in = (4 * 4 * 16 * 4 * 8 * 10 ** 9) // 10 ** 6 + 1000
+    t_out = (2 * 2 * 4 * 6 * 4 * 16 * 10 ** 9) // 10 ** 6 + 1000
+    assert cost == t_in + t_con + t_out
+    # the same layer with 7 x 7 kernels: m = 2 -> alpha 8 (8 quarters), m = 4 -> alpha 10 (9), m = 6 -> alpha 12 (16)
+    L7 = T.Layer(1, 8, 16, 12, 12, 7, 1, 3)
+    for m, quarters in ((2, 8), (4, 9), (6, 16)):
+        alpha = m + 6
+        tiles = (12 // m) ** 2
+        _, _, cost = T.winograd_cost(L7, m, T.OPERAND_TF32, 1, cal)
+        items = alpha * alpha                              # 1 tile block, 1 channel block
+        rounds_sms = -(-items // 7) * 7
+        t_in = (quarters * alpha * alpha * alpha * tiles * 8 * 10 ** 9) // 10 ** 6 + 1000
+        t_con = (2 * alpha * alpha * 16 * 8 * tiles * 10 ** 9 // items * rounds_sms) // 10 ** 6 + 1000
+        t_out = (2 * m * alpha * (alpha + m) * tiles * 16 * 10 ** 9) // 10 ** 6 + 1000
+        assert cost == t_in + t_con + t_out, m
+
+
 def test_fused_cost_by_hand():
     L = T.Layer(2, 64, 256, 8, 8, 3, 1, 1)                 # 32 tiles: 1 tile block, 2 channel blocks, 2 K blocks
     x, y, u = 4 * 2 * 64 * 64, 4 * 2 * 256 * 64, 16 * 256 * 64 * 4
