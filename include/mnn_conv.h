@@ -63,7 +63,9 @@ enum { MNN_STAGE_WEIGHT = 1, MNN_STAGE_INPUT = 2, MNN_STAGE_CONTRACT = 4, MNN_ST
 /*
  * Options of mnn_conv_plan_ex.  Zero-initialise for the defaults of mnn_conv_plan
  * except `relu`, which mnn_conv_plan sets to 1.
- *   groups     1, or Cin (= Cout) for a depthwise layer.  0 means 1.
+ *   groups     any divisor of Cin and Cout (w is [Cout][Cin/groups][k][k]).  1: all schemes; Cin = Cout = groups
+ *              (depthwise 3x3, padding 1, stride 1 or 2): the depthwise kernels; every other grouped layer runs the
+ *              generic sliding-window kernel.  0 means 1.
  *   relu       0/1: y = max(0, .) after the bias.
  *   precision  accuracy class the result must meet against an exact evaluation:
  *              MNN_PREC_TF32: relative L2 error <= 1e-3; MNN_PREC_BF16: <= 1e-2.
@@ -328,7 +330,7 @@ typedef struct mnn_net_s* mnn_net_t;
 
 typedef struct {
     int Cin, Cout, k, stride, pad, dilation;
-    int groups;        /* 0 or 1, or Cin (= Cout) for depthwise */
+    int groups;        /* 0 or 1, Cin (= Cout) for depthwise, or any divisor of Cin and Cout */
     int relu;
 } mnn_layer_desc;
 

@@ -205,10 +205,6 @@ mnn_conv_plan_t mnn_conv_plan_ex(int N, int Cin, int Cout, int H, int W, int k, 
         fail(MNN_EINVAL, "groups must divide Cin and Cout");
         return nullptr;
     }
-    if (o.groups != 1 && !(o.groups == Cin && Cin == Cout)) {
-        fail(MNN_EUNSUPPORTED, "groups must be 1 or Cin = Cout (depthwise)");
-        return nullptr;
-    }
     if (o.precision != MNN_PREC_TF32 && o.precision != MNN_PREC_BF16) {
         fail(MNN_EINVAL, "precision must be MNN_PREC_TF32 or MNN_PREC_BF16");
         return nullptr;

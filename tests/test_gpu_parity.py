@@ -393,7 +393,8 @@ def test_depthwise_even_widths(torch, C, H, W_, N, stride):
 
 @pytest.mark.parametrize("Cin,Cout,H,k,stride,pad,dil,groups", [
     (3, 32, 32, 3, 2, 1, 1, 1), (3, 16, 30, 7, 2, 3, 1, 1), (6, 6, 9, 3, 1, 1, 2, 6), (5, 7, 8, 2, 1, 0, 1, 1),
-    (4, 4, 6, 5, 3, 2, 1, 4), (3, 40, 37, 3, 2, 1, 1, 1), (3, 24, 19, 3, 1, 1, 1, 1), (3, 33, 50, 3, 2, 0, 1, 1)])
+    (4, 4, 6, 5, 3, 2, 1, 4), (16, 64, 11, 2, 1, 0, 2, 4), (32, 8, 14, 3, 2, 0, 1, 2), (8, 32, 13, 1, 1, 0, 1, 2),
+    (64, 4, 9, 2, 2, 1, 2, 4), (3, 40, 37, 3, 2, 1, 1, 1), (3, 24, 19, 3, 1, 1, 1, 1), (3, 33, 50, 3, 2, 0, 1, 1)])
 def test_generic_direct(torch, Cin, Cout, H, k, stride, pad, dil, groups):
     layer = W.ConvLayer("t", 2, Cin, Cout, H, H, k, stride, pad, dil, groups=groups, relu=True, seed=k)
     x, w, b = W.make_inputs(layer)
