@@ -370,7 +370,7 @@ def time_workload(state, steps, warmup, launch, flush, dev, dist, barrier, sampl
     stage_ms = {n: 0.0 for n in stage_names}
     stage_n = {n: 0 for n in stage_names}
     stage_bytes = {n: 0 for n in stage_names}
-    tensor_flops, tensor_roof_s = 0.0, 0.0          # executed MMA flops and the time the measured peak would need
+    tensor_flops, tensor_roof_s, tensor_roof_burst_s = 0.0, 0.0, 0.0   # executed MMA flops; the time the measured peaks would need
     peaks = measured_peaks()
     per_layer = []
     prof_steps = min(steps, 200)
@@ -390,9 +390,10 @@ def time_workload(state, steps, warmup, launch, flush, dev, dist, barrier, sampl
                     stage_bytes[nm] += work[nm]["bytes"]
             if info.algo != B.ALGO_DIRECT and n[2]:
                 fl = work["contraction"]["flops"]
-                peak = peaks["bf16_tflops"] * (1.0 if info.operand == B.OPERAND_BF16 else TF32_OVER_BF16)
+                ratio = 1.0 if info.operand == B.OPERAND_BF16 else TF32_OVER_BF16
                 tensor_flops += fl
-                tensor_roof_s += fl / (peak * 1e12)
+                tensor_roof_s += fl / (peaks["bf16_tflops_sustained"] * ratio * 1e12)
+                tensor_roof_burst_s += fl / (peaks["bf16_tflops"] * ratio * 1e12)
             if k == prof_steps - 1:
                 per_layer.append({"name": s["layer"].name, "algo": B.ALGO_NAMES[info.algo], "m": info.m,
                                   "operand": B.OPERAND_NAMES[info.operand], "passes": info.passes, "fused": info.fused,
@@ -415,14 +416,19 @@ def time_workload(state, steps, warmup, launch, flush, dev, dist, barrier, sampl
         sec = stage_ms["contraction"] * 1e-3
         stages["contraction"]["tensor_TFLOPs"] = tensor_flops / sec / 1e12
         stages["contraction"]["frac_of_tensor_peak"] = tensor_roof_s / sec
+        stages["contraction"]["frac_of_burst_tensor_peak"] = tensor_roof_burst_s / sec
     dominant = max(stages, key=lambda n: stages[n]["ms_per_step"])
     d = stages[dominant]
     if dominant == "contraction" and d.get("frac_of_tensor_peak", 0.0) >= d["frac_of_hbm"]:
-        # the dense contraction against the measured tensor peak of each layer's operand format (burst figure: the
-        # kernel is timed alone by its own events); TF32 = measured BF16 x the nominal ratio 1.1 / 2.25
+        # the dense contraction against the measured tensor peak of each layer's operand format; TF32 = measured
+        # BF16 x the nominal ratio 1.1 / 2.25.  The launches are timed by their own events but inside a run of
+        # seconds under the power cap (see "clocks"), so the denominator is the SUSTAINED figure; the fraction of
+        # the burst figure is printed beside it
         roofline = {"kernel": dominant, "bound": "tensor", "achieved": d["tensor_TFLOPs"],
                     "peak": d["tensor_TFLOPs"] / d["frac_of_tensor_peak"], "unit": "TFLOP/s",
-                    "frac": d["frac_of_tensor_peak"]}
+                    "frac": d["frac_of_tensor_peak"], "peak_kind": "sustained (power-capped loop)",
+                    "peak_burst": d["tensor_TFLOPs"] / d["frac_of_burst_tensor_peak"],
+                    "frac_of_burst": d["frac_of_burst_tensor_peak"]}
     else:
         roofline = {"kernel": dominant, "bound": "hbm", "achieved": d["algorithmic_GBps"], "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": d["frac_of_hbm"]}
