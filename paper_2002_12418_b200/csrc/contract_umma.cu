@@ -8,7 +8,8 @@
 // buffered), four warps drain the accumulator with tcgen05.ld and store it (one per
 // quarter of the tensor-memory lanes, the load of the next 16 columns in flight while
 // the previous 16 are stored; two warps per quarter, each taking half of the columns,
-// were measured and gained nothing: the stores already run near the HBM write rate).
+// gain nothing on long K loops, where the stores already run near the HBM write rate,
+// and are used where the K loop is at most two blocks long).
 // The MMA "M" dimension is the tile index t (operand A = V), "N" the output channel
 // (operand B = U), "K" the input channel; TF32 or BF16 operands, fp32 accumulation;
 // with passes = 3 the operands come as hi + lo pairs and hi*hi + lo*hi + hi*lo are
@@ -39,8 +40,11 @@ namespace mnnb {
 
 namespace {
 
-constexpr int kEpilogueWarps = 4;      // a multiple of 4: warps per quarter of the lanes split the columns
-constexpr int kThreads = 64 + 32 * kEpilogueWarps;   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
+// warp 0: TMA, warp 1: MMA + TMEM owner, then 4 or 8 epilogue warps (KernelParams::epi_warps; the warps of a
+// lane quarter split the columns).  Eight pay where the K loop is one or two blocks long and the epilogue
+// decides (a 32 -> 64 pointwise layer at 112 x 112: 78 -> 68 us); on long K loops they cost 0.3-0.6 %.
+constexpr int kMaxEpilogueWarps = 8;
+constexpr int kMaxThreads = 64 + 32 * kMaxEpilogueWarps;
 constexpr int kTileM = 128;            // tiles (rows of V) per work item
 constexpr int kMaxStages = 8;
 constexpr int kMaxSharedBias = 2048;    // output channels whose bias is staged in shared memory (+ 16 of slack)
@@ -60,6 +64,7 @@ struct KernelParams {
     // 1: hi and lo operand tiles arrive with one copy each for V and U (maps with a hi / lo dimension, see
     // encode_operand_pair_map); halves the copies the producer issues per stage
     int merged;
+    int epi_warps;     // 4 or 8 (the block has 64 + 32 * epi_warps threads)
 };
 
 // status codes written on a bounded wait that ran out
@@ -83,7 +88,7 @@ __device__ __forceinline__ uint64_t desc_k(uint32_t smem_addr)
 // would leave room for two pipeline stages only (hi + lo operands with wide channel blocks): the same bytes
 // in flight in twice as many stages keep the tensor core fed across the TMA latency.
 template <int KIND, int SW>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMaxThreads, 1)
 contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_constant__ CUtensorMap map_v_lo,
                      const __grid_constant__ CUtensorMap map_u_hi, const __grid_constant__ CUtensorMap map_u_lo,
                      const __grid_constant__ CUtensorMap map_x_ragged, KernelParams p)
@@ -116,7 +121,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(ptx::smem_u32(&tfull_bar[s]), 1);
-            ptx::mbar_init(ptx::smem_u32(&tempty_bar[s]), kEpilogueWarps);
+            ptx::mbar_init(ptx::smem_u32(&tempty_bar[s]), (uint32_t)p.epi_warps);
         }
         abort_flag = 0;
         ptx::fence_barrier_init();
@@ -135,8 +140,8 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     ptx::grid_dependency_wait();
     const bool bias_in_smem = p.epi.mode == 1 && p.Cout <= kMaxSharedBias;
     if (bias_in_smem && warp >= 2) {
-        for (int i = threadIdx.x - 64; i < p.Cout; i += kThreads - 64) s_bias[i] = p.epi.bias ? __ldg(p.epi.bias + i) : 0.0f;
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");          // the epilogue warps only
+        for (int i = threadIdx.x - 64; i < p.Cout; i += 32 * p.epi_warps) s_bias[i] = p.epi.bias ? __ldg(p.epi.bias + i) : 0.0f;
+        asm volatile("bar.sync 1, %0;" ::"r"(32 * p.epi_warps) : "memory");             // the epilogue warps only
     }
 
     const int k_elems = (KIND == 0 ? 32 : 64) * SW / 128;   // elements of K per shared-memory row
@@ -287,7 +292,7 @@ contract_umma_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 dst = p.epi.y + ((size_t)img * p.Cout + co0) * p.epi.ohw + (t_ok ? t - img * p.epi.ohw : 0);
             }
             // this warp's chunks of 16 columns
-            constexpr int kParts = kEpilogueWarps / 4;
+            const int kParts = p.epi_warps >> 2;
             const int n_chunks = (n_co + 15) >> 4;
             const int per_part = (n_chunks + kParts - 1) / kParts;
             const int ch_begin = min(part * per_part, n_chunks), ch_end = min(ch_begin + per_part, n_chunks);
@@ -661,7 +666,8 @@ cudaError_t launch_contract_umma_x(const UmmaContract& uc, const float* x, const
     p.epi = epi;
     p.status = status;
     const long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
-    return launch_overlapped(contract_umma_kernel<0, 128>, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream,
+    p.epi_warps = uc.k_blocks <= 2 ? 8 : 4;
+    return launch_overlapped(contract_umma_kernel<0, 128>, dim3((unsigned)grid), dim3(64 + 32 * p.epi_warps), (size_t)uc.smem_bytes, stream,
                              map_lead, map_last, uc.map_u_hi, uc.map_u_lo, map_ragged, p);
 }
 
@@ -694,7 +700,8 @@ cudaError_t launch_contract_umma(const UmmaContract& uc, long long tiles, const 
     long long grid = p.n_items < uc.num_sms ? p.n_items : uc.num_sms;
     auto kern = uc.kind == 0 ? (uc.stages_sw == 64 ? contract_umma_kernel<0, 64> : contract_umma_kernel<0, 128>)
                              : (uc.stages_sw == 64 ? contract_umma_kernel<1, 64> : contract_umma_kernel<1, 128>);
-    return launch_overlapped(kern, dim3((unsigned)grid), dim3(kThreads), (size_t)uc.smem_bytes, stream, uc.map_v_hi,
+    p.epi_warps = (uc.alpha2 == 1 && uc.k_blocks <= 2) ? 8 : 4;
+    return launch_overlapped(kern, dim3((unsigned)grid), dim3(64 + 32 * p.epi_warps), (size_t)uc.smem_bytes, stream, uc.map_v_hi,
                              uc.map_v_lo, uc.map_u_hi, uc.map_u_lo, uc.map_u_hi, p);
 }
 
