@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmnnconv_b200.so")
-SOURCES = ["api.cu", "calibrate.cu", "contract_umma.cu", "wino_fused.cu", "strassen.cu", "implicit_gemm.cu", "wino_rect.cu", "gather_direct.cu", "wino_transforms.cu", "wino_inst_k2.cu", "wino_inst_a4_6.cu",
+SOURCES = ["api.cu", "calibrate.cu", "contract_umma.cu", "contract_pair.cu", "wino_fused.cu", "strassen.cu", "implicit_gemm.cu", "wino_rect.cu", "gather_direct.cu", "wino_transforms.cu", "wino_inst_k2.cu", "wino_inst_a4_6.cu",
            "wino_inst_a8.cu", "wino_inst_a10.cu", "wino_inst_a12.cu",
            "generator.cpp", "planner.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -11,6 +12,7 @@
 #include "../../include/mnn_conv.h"
 #include "generator.h"
 #include "implicit_gemm.h"
+#include "contract_pair.h"
 #include "contract_umma.h"
 #include "kernels.h"
 #include "planner.h"
@@ -62,6 +64,8 @@ struct mnn_conv_plan_s {
     long long ws_bytes = 0;
     const float* prepared_w = nullptr;
     UmmaContract uc;
+    PairContract pc;           // the Winograd contraction on pairs of SMs, when use_pair
+    bool use_pair = false;
     bool strassen = false;           // GEMM scheme through one Strassen level: seven half-size products
     int rect = 0;                    // 1: kernel 1 x k, 2: kernel k x 1 (one-dimensional Winograd along the long axis)
     int pad_h = 0, pad_w = 0;        // rectangular plans: padding per axis (s.pad is unused there)
@@ -434,6 +438,20 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     return MNN_OK;
 }
 
+// Whether the Winograd contraction of a layer runs on pairs of SMs (256 x 256 blocks per work item): at least 256
+// output channels and at least two work items per SM pair, so that the coarser items still fill the machine.
+// MNN_CONV_PAIR=0 in the environment keeps the single-SM kernel (for comparisons).
+static bool pair_contraction_wanted(int Cout, long long tiles, int alpha2)
+{
+    static const bool off = [] {
+        const char* v = std::getenv("MNN_CONV_PAIR");
+        return v && v[0] == '0';
+    }();
+    if (off || Cout < 256) return false;
+    const long long items = ((tiles + 255) / 256) * ((Cout + 255) / 256) * alpha2;
+    return items >= 148;
+}
+
 // Tensor maps and launch parameters of the plan's tensor-core kernel for the workspace now in p->ws / p->tws.
 static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
 {
@@ -451,8 +469,16 @@ static cudaError_t setup_tensor_kernels(mnn_conv_plan_t p, const char** why)
         return implicit_gemm_setup(&p->ig, g, s.Cout, u_hi(p), why);
     }
     if (p->gemm_x) return umma_contract_setup_x(&p->uc, p->s.Cout, p->s.Cin, p->cin_pad, p->s.N, p->s.H * p->s.W, u_hi(p), why);
-    return umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
-                               v_lo(p), why);
+    cudaError_t e = umma_contract_setup(&p->uc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p),
+                                        v_hi(p), v_lo(p), why);
+    p->use_pair = false;
+    if (e == cudaSuccess && alpha2 > 1 && pair_contraction_wanted(p->s.Cout, p->chunk_tiles, alpha2)) {
+        const char* why_not = nullptr;
+        if (pair_contract_setup(&p->pc, p->store_mode, alpha2, p->s.Cout, p->cin_pad, p->chunk_tiles, u_hi(p), u_lo(p), v_hi(p),
+                                v_lo(p), &why_not) == cudaSuccess)
+            p->use_pair = true;
+    }
+    return e;
 }
 
 // Workspace in two parts (used by the network plan): `persistent` holds the status word and U
@@ -731,6 +757,8 @@ int mnn_conv_run_stages(mnn_conv_plan_t p, const float* x, const float* w, const
             if (reference)
                 e = launch_contract_reference(u_hi(p), u_lo(p), v_hi(p), v_lo(p), p->store_mode, alpha2, s.Cout, g.tiles,
                                               p->cin_pad, (long long)s.Cout * p->cin_pad, g.v_plane, epi, st);
+            else if (p->use_pair)
+                e = launch_contract_pair(p->pc, g.tiles, m_buf(p), p->m_row_stride, status_word(p), st);
             else
                 e = launch_contract_umma(p->uc, g.tiles, epi, status_word(p), st);
             if (e != cudaSuccess) return fail_cuda(e, "Winograd contraction");

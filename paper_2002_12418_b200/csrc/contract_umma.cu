@@ -419,8 +419,8 @@ EncodeTiledFn get_encode_fn()
 }  // namespace
 
 // 3-D map over [planes][rows][k] (k contiguous), box = [1][box_rows][128 bytes of k], 128-byte swizzle.
-static bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
-                                  long long plane_stride_elems, int box_rows, int sw);
+bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
+                           long long plane_stride_elems, int box_rows, int sw);
 
 bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
                         long long plane_stride_elems, int box_rows)
@@ -429,8 +429,8 @@ bool encode_operand_map(CUtensorMap* map, void* base, int elem_bytes, long long 
 }
 
 // The same with rows of `sw` bytes (128 or 64) and the matching swizzle.
-static bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
-                                  long long plane_stride_elems, int box_rows, int sw)
+bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
+                           long long plane_stride_elems, int box_rows, int sw)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
@@ -447,8 +447,8 @@ static bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, 
 
 // 4-D map over a hi / lo operand pair: [planes][hi, lo][rows][k], the lo array `lo_offset_bytes` behind the hi
 // array; box = [1][2][box_rows][sw bytes of k].  One copy lands the hi tile and, right behind it, the lo tile.
-static bool encode_operand_pair_map(CUtensorMap* map, void* base_hi, long long lo_offset_bytes, int elem_bytes, long long k_len,
-                                    long long rows, long long planes, long long plane_stride_elems, int box_rows, int sw)
+bool encode_operand_pair_map(CUtensorMap* map, void* base_hi, long long lo_offset_bytes, int elem_bytes, long long k_len,
+                             long long rows, long long planes, long long plane_stride_elems, int box_rows, int sw)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn || lo_offset_bytes <= 0 || lo_offset_bytes % 16 != 0 || lo_offset_bytes >= (1ll << 40)) return false;

@@ -27,6 +27,14 @@ struct UmmaContract {
     int merged = 0;                    // hi and lo tiles of an operand arrive with one copy (maps with a hi / lo dimension)
     bool ready = false;
 };
+// Tensor maps over an operand array [planes][rows][k] (k contiguous): box = [1][box_rows][sw bytes of k] with the
+// sw-byte swizzle (sw = 128 or 64); and over a hi / lo pair of such arrays (the lo array lo_offset_bytes behind the hi
+// array): box = [1][2][box_rows][sw bytes], the hi tile landing first, the lo tile right behind it.
+bool encode_operand_map_sw(CUtensorMap* map, void* base, int elem_bytes, long long k_len, long long rows, long long planes,
+                           long long plane_stride_elems, int box_rows, int sw);
+bool encode_operand_pair_map(CUtensorMap* map, void* base_hi, long long lo_offset_bytes, int elem_bytes, long long k_len,
+                             long long rows, long long planes, long long plane_stride_elems, int box_rows, int sw);
+
 // Encodes the tensor maps for U/V at the given device addresses.  Returns a CUDA error or cudaSuccess;
 // *why gets a static reason on failure.
 cudaError_t umma_contract_setup(UmmaContract* uc, int mode, int alpha2, int Cout, int cin_pad, long long tiles_capacity,
