@@ -438,7 +438,7 @@ int mnn_conv_plan_query(mnn_conv_plan_t p, mnn_conv_info* info)
     return MNN_OK;
 }
 
-// Whether the Winograd contraction of a layer runs on pairs of SMs (256 x 256 blocks per work item): at least 256
+// Whether the Winograd contraction of a layer runs on pairs of SMs (256 tiles x 256 channels per work item): at least 256
 // output channels and at least two work items per SM pair, so that the coarser items still fill the machine.
 // MNN_CONV_PAIR=0 in the environment keeps the single-SM kernel (for comparisons).
 static bool pair_contraction_wanted(int Cout, long long tiles, int alpha2)
@@ -447,7 +447,7 @@ static bool pair_contraction_wanted(int Cout, long long tiles, int alpha2)
         const char* v = std::getenv("MNN_CONV_PAIR");
         return v && v[0] == '0';
     }();
-    if (off || Cout < 256) return false;
+    if (off || Cout < 256) return false;     // narrower layers measured slower on pairs (128 channels: 44 -> 63 us)
     const long long items = ((tiles + 255) / 256) * ((Cout + 255) / 256) * alpha2;
     return items >= 148;
 }

@@ -28,13 +28,14 @@ namespace {
 
 constexpr int kPairThreads = 192;
 constexpr int kRows = 128;             // rows of V, and rows of U, per CTA and stage
-constexpr int kPairN = 256;            // output channels per work item (MMA N)
+constexpr int kPairMaxN = 256;         // output channels per work item (MMA N): PairParams::bn, a multiple of 32
 constexpr int kPairMaxStages = 8;
 constexpr int kPairSmemBudget = 200 * 1024;
 constexpr int kErrPairProducer = 21, kErrPairMmaFull = 22, kErrPairMmaTmem = 23, kErrPairEpilogue = 24;
 
 struct PairParams {
     int alpha2, n_row_blocks, n_co_blocks, k_blocks, passes, stages, Cout, merged;
+    int bn;            // output channels per work item; each CTA stages bn / 2 rows of U
     long long tiles, n_items;
     float* M;
     long long m_row_stride;
@@ -156,8 +157,9 @@ contract_pair_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t tile_bytes = kRows * SW;
     const uint32_t split = p.passes == 3 ? 2u : 1u;
-    const uint32_t stage_bytes = 2u * tile_bytes * split;            // [A_hi][A_lo?][B_hi][B_lo?]
-    const uint32_t off_a_lo = tile_bytes, off_b_hi = tile_bytes * split, off_b_lo = tile_bytes * split + tile_bytes;
+    const uint32_t b_bytes = (uint32_t)(p.bn / 2) * SW;              // this CTA's half of the U tile
+    const uint32_t stage_bytes = (tile_bytes + b_bytes) * split;     // [A_hi][A_lo?][B_hi][B_lo?]
+    const uint32_t off_a_lo = tile_bytes, off_b_hi = tile_bytes * split, off_b_lo = tile_bytes * split + b_bytes;
     volatile int* abortp = &abort_flag;
 
     if (threadIdx.x == 0) {
@@ -197,7 +199,7 @@ contract_pair_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                 const long long r = item / p.n_row_blocks;
                 const int nb = (int)(r % p.n_co_blocks);
                 const int xi = (int)(r / p.n_co_blocks);
-                const int v_row = (rb * 2 + (int)rank) * kRows, u_row = nb * kPairN + (int)rank * kRows;
+                const int v_row = (rb * 2 + (int)rank) * kRows, u_row = nb * p.bn + (int)rank * (p.bn / 2);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, abortp)) {
                         if (!*abortp) atomicCAS(p.status, 0, kErrPairProducer);
@@ -229,7 +231,7 @@ contract_pair_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            const uint32_t idesc = ptx::mma_idesc(KIND == 0 ? 2 : 1, 2 * kRows, kPairN);
+            const uint32_t idesc = ptx::mma_idesc(KIND == 0 ? 2 : 1, 2 * kRows, p.bn);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             for (long long item = pair; item < p.n_items && ok; item += n_pairs) {
@@ -240,7 +242,7 @@ contract_pair_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
                     break;
                 }
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * (uint32_t)kPairN;
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)kPairMaxN;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full_bar[stage]), phase, abortp)) {
                         if (!*abortp) atomicCAS(p.status, 0, kErrPairMmaFull);
@@ -297,9 +299,9 @@ contract_pair_kernel(const __grid_constant__ CUtensorMap map_v_hi, const __grid_
             ptx::tc_fence_after();
             const long long t = ((long long)rb * 2 + rank) * kRows + q * 32 + lane;     // this thread's tile
             const bool t_ok = t < p.tiles;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)kPairN;
-            const int co0 = nb * kPairN;
-            const int n_co = min(kPairN, p.Cout - co0);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)kPairMaxN;
+            const int co0 = nb * p.bn;
+            const int n_co = min(p.bn, p.Cout - co0);
             float* dst = p.M + ((size_t)xi * p.Cout + co0) * p.m_row_stride + (t_ok ? t : 0);
             const int n_chunks = (n_co + 15) >> 4;
             uint32_t va[16], vb[16];
@@ -381,11 +383,12 @@ cudaError_t pair_contract_setup(PairContract* pc, int mode, int alpha2, int Cout
     // rows of 128 bytes unless hi + lo stages of that size leave fewer than four (then 64-byte rows, when the K
     // loop is long enough)
     int sw = 128;
-    if ((kPairSmemBudget - 1024) / (2 * kRows * sw * split) < 4 && cin_pad * eb >= 4 * 64) sw = 64;
+    pc->bn = Cout >= kPairMaxN ? kPairMaxN : (Cout + 31) / 32 * 32;
+    if ((kPairSmemBudget - 1024) / ((kRows + pc->bn / 2) * sw * split) < 4 && cin_pad * eb >= 4 * 64) sw = 64;
     pc->sw = sw;
     const int k_elems = sw / eb;
     pc->k_blocks = (cin_pad + k_elems - 1) / k_elems;
-    int stages = (kPairSmemBudget - 1024) / (2 * kRows * sw * split);
+    int stages = (kPairSmemBudget - 1024) / ((kRows + pc->bn / 2) * sw * split);
     if (stages > kPairMaxStages) stages = kPairMaxStages;
     if (stages < 2) {
         *why = "shared memory cannot hold two pipeline stages";
@@ -399,7 +402,7 @@ cudaError_t pair_contract_setup(PairContract* pc, int mode, int alpha2, int Cout
     if (split == 2) {
         const long long dv = static_cast<char*>(V_lo) - static_cast<char*>(V_hi), du = static_cast<char*>(U_lo) - static_cast<char*>(U_hi);
         if (encode_operand_pair_map(&pc->map_v_hi, V_hi, dv, eb, cin_pad, tiles_capacity, alpha2, v_plane, kRows, sw) &&
-            encode_operand_pair_map(&pc->map_u_hi, U_hi, du, eb, cin_pad, Cout, alpha2, u_plane, kRows, sw)) {
+            encode_operand_pair_map(&pc->map_u_hi, U_hi, du, eb, cin_pad, Cout, alpha2, u_plane, pc->bn / 2, sw)) {
             pc->merged = 1;
             pc->map_v_lo = pc->map_v_hi;
             pc->map_u_lo = pc->map_u_hi;
@@ -407,10 +410,10 @@ cudaError_t pair_contract_setup(PairContract* pc, int mode, int alpha2, int Cout
     }
     if (!pc->merged) {
         ok = encode_operand_map_sw(&pc->map_v_hi, V_hi, eb, cin_pad, tiles_capacity, alpha2, v_plane, kRows, sw) &&
-             encode_operand_map_sw(&pc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, kRows, sw);
+             encode_operand_map_sw(&pc->map_u_hi, U_hi, eb, cin_pad, Cout, alpha2, u_plane, pc->bn / 2, sw);
         if (ok && split == 2)
             ok = encode_operand_map_sw(&pc->map_v_lo, V_lo, eb, cin_pad, tiles_capacity, alpha2, v_plane, kRows, sw) &&
-                 encode_operand_map_sw(&pc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, kRows, sw);
+                 encode_operand_map_sw(&pc->map_u_lo, U_lo, eb, cin_pad, Cout, alpha2, u_plane, pc->bn / 2, sw);
         if (ok && split == 1) {
             pc->map_v_lo = pc->map_v_hi;
             pc->map_u_lo = pc->map_u_hi;
@@ -438,7 +441,8 @@ cudaError_t launch_contract_pair(const PairContract& pc, long long tiles, float*
     PairParams p;
     p.alpha2 = pc.alpha2;
     p.n_row_blocks = (int)((tiles + 2 * kRows - 1) / (2 * kRows));
-    p.n_co_blocks = (pc.Cout + kPairN - 1) / kPairN;
+    p.bn = pc.bn;
+    p.n_co_blocks = (pc.Cout + pc.bn - 1) / pc.bn;
     p.k_blocks = pc.k_blocks;
     p.passes = pc.passes;
     p.stages = pc.stages;

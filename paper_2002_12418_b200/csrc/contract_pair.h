@@ -11,6 +11,7 @@ struct PairContract {
     int passes = 1;        // 1 or 3 (hi + lo operands)
     int alpha2 = 0, Cout = 0, cin_pad = 0;
     long long tiles_capacity = 0;
+    int bn = 256;          // output channels per work item (MMA N, a multiple of 32, at most 256)
     int k_blocks = 0, stages = 0, sw = 128, merged = 0, num_sms = 0, smem_bytes = 0;
     bool ready = false;
 };

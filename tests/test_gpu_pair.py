@@ -34,6 +34,7 @@ def run(torch, layer, opts, inputs):
     (8, 64, 300, 40, 5, 4, "tf32", 3),        # two channel blocks, the second of 44 channels; TF32 hi + lo
     (12, 128, 512, 30, 3, 2, "tf32", 1),      # single-pass TF32, 2700 tiles: the last block's second CTA is empty
     (10, 128, 256, 48, 3, 2, "bf16", 1),      # single-pass BF16 (128-byte rows of 64 elements)
+    (6, 64, 288, 44, 3, 4, "bf16", 3),        # 288 channels: a second block of 32, 121 tiles per image
 ])
 def test_pair_contraction_parity(N, Cin, Cout, H, k, m, operand, passes):
     import torch
