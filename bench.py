@@ -37,10 +37,10 @@ UNIT = "TFLOP/s"
 NCU_DRAM_TRAFFIC = {
     "config4_b64/tf32": {
         "plans": [("winograd", 4, "bf16", 3), ("winograd", 4, "bf16", 3), ("winograd", 4, "bf16", 3), ("winograd", 4, "tf32", 3)],
-        # mean over the four contraction launches of one step, captured at batch 16 (190.4 / 456.4 / 29.9 / 99.7 MB;
-        # taken with the current kernel: one copy per hi+lo operand pair, epilogue warps chosen per launch)
+        # mean over the four contraction launches of one step, captured at batch 16 (188.9 / 453.1 / 29.9 / 99.5 MB;
+        # taken with the current kernels: the two 3x3 layers on pairs of SMs, the 128-channel layers on single SMs)
         # and multiplied by four; at batch 64 less of V and M stays in L2, so the true figure is somewhat higher
-        "contraction": 4 * 193.8e6,
+        "contraction": 4 * 192.4e6,
         "source": "stored ncu capture of the batch-16 copy of this workload, scaled by 4; not measured by this run",
     },
 }
