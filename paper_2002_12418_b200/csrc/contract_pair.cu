@@ -31,7 +31,7 @@ constexpr int kRows = 128;             // rows of V, and rows of U, per CTA and 
 constexpr int kPairMaxN = 256;         // output channels per work item (MMA N): PairParams::bn, a multiple of 32
 constexpr int kPairMaxStages = 8;
 constexpr int kPairSmemBudget = 200 * 1024;
-constexpr int kErrPairProducer = 21, kErrPairMmaFull = 22, kErrPairMmaTmem = 23, kErrPairEpilogue = 24;
+constexpr int kErrPairProducer = 41, kErrPairMmaFull = 42, kErrPairMmaTmem = 43, kErrPairEpilogue = 44;   // status codes
 
 struct PairParams {
     int alpha2, n_row_blocks, n_co_blocks, k_blocks, passes, stages, Cout, merged;
