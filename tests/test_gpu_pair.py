@@ -61,3 +61,15 @@ def test_pair_contraction_exact_on_integers():
     for _ in range(2):
         got = run(torch, layer, opts, inputs)
         assert np.array_equal(got.astype(np.float64), ref)
+
+def test_pair_contraction_in_chunks():
+    """A run split into chunks of images whose last chunk is smaller: the pair kernel then gets fewer tiles than its
+    tensor maps were made for, and every chunk must still equal the oracle."""
+    import torch
+    B.lib()
+    layer = W.ConvLayer("t", 25, 64, 256, 40, 40, 3, 1, 1, 1, relu=True, seed=11)
+    inputs = W.make_inputs(layer)
+    opts = B.make_opts(relu=True, force_algo=B.ALGO_WINOGRAD, force_m=4, operand=B.OPERAND_BF16, passes=3, chunk_images=11)
+    got = run(torch, layer, opts, inputs)                 # chunks of 11, 11 and 3 images: 1100 / 1100 / 300 tiles (180 work items per full chunk)
+    ref = oc.direct_conv(*inputs, 1, 1, 1, 1, True)
+    assert_close(got, ref, B.PREC_TF32, "pair contraction in chunks")
