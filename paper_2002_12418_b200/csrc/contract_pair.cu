@@ -6,7 +6,8 @@
 // channels), the tensor cores of both SMs read both halves, and each CTA's tensor memory receives the 128 x 256
 // accumulator of its own rows.  Per output a CTA therefore pulls 2 x 128 operand rows per K block from L2
 // instead of 128 + 256: two thirds of the single-CTA kernel's traffic, which is what bounds that kernel (its
-// shared memory holds 4 stages x 48 KB against a round trip of about 3 us; here 6 stages x 32 KB).
+// shared memory holds 4 stages x 48 KB against a round trip of about 3 us; here 6 stages x 32 KB, or 3 x 64 KB
+// with 128-byte rows on long K loops).
 //
 // Roles per CTA as in contract_umma.cu (warp 0 lane 0: TMA producer, warp 1: tensor memory and, in the cluster's
 // first CTA only, the MMA issue, warps 2-5: epilogue).  Barriers: the "operands landed" barriers that count
